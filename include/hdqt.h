@@ -1,0 +1,253 @@
+/*
+ * hdqt.h - C ABI of the B200 (sm_100a) HDQT quantized training GEMM library.
+ *
+ * HDQT = Hadamard Domain Quantized Training (arXiv 2310.03675).  The library
+ * implements the paper's quantized matrix multiply Z = X W (Section 3) for the
+ * forward product and the two backward products:
+ *
+ *   1. block-diagonal Sylvester Hadamard transform along the contraction
+ *      dimension of both operands (Section 3, "BlockDiag(H_k, ..., H_k)");
+ *   2. max-calibrated uniform integer quantizer Q (Section 3, definition of Q),
+ *      with stochastic rounding on the tensors the paper singles out
+ *      (Section 3, sensitivity paragraph) and the 0.975 clip on the forward
+ *      operands (Section 4, hyper-parameters);
+ *   3. integer matrix multiply whose contraction is cut into tiles of s terms,
+ *      each tile sum held in a low-bit accumulator (Section 3, "tiled
+ *      quantization ... tiles of size s"; Section 4, "block-size for
+ *      accumulators (32)"; Section 4.2, "8-bit integer accumulators in forward
+ *      and backward-pass");
+ *   4. wide sum of the tile results and a dequantising scale; no inverse
+ *      transform is needed because H H^T = n I (Section 3).
+ *
+ * Conventions that hold for every entry point
+ *   - Every pointer is a DEVICE pointer owned by the caller unless it is
+ *     marked "host".  The library allocates no device memory, keeps no pointer
+ *     after the call returns, and never synchronises the host: all work is
+ *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *     default stream).
+ *   - Return value: HDQT_OK, or an error detected on the host before anything
+ *     was launched (nothing is launched in that case).
+ *   - Errors only the device can see (a non-finite input, a bounded wait that
+ *     ran out) are recorded in *dev_status (device int32, sticky maximum of
+ *     hdqt_status_t values; the caller zeroes it and reads it after a
+ *     synchronise).  dev_status may be NULL (such errors are then dropped).
+ *   - Alignment: src / out pointers 16 bytes; code buffers and workspaces
+ *     128 bytes.
+ *   - Code layout: int8 lanes, row-major [rows, K_pad] with the contraction
+ *     index contiguous, K_pad = hdqt_padded_k(K, had_block); padded entries are
+ *     codes of zero-padded source entries.
+ *   - Floating point: every step is IEEE binary32, round-to-nearest-even, no
+ *     fused multiply-add; integer results are exact and reproducible bit for
+ *     bit for a given (seed, tag).
+ */
+#ifndef HDQT_H_
+#define HDQT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  HDQT_OK = 0,
+  HDQT_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, bad enum      */
+  HDQT_ERR_UNSUPPORTED = 2,  /* valid in the paper's terms, not built here     */
+  HDQT_ERR_ALIGNMENT = 3,    /* pointer or leading dimension not aligned       */
+  HDQT_ERR_WORKSPACE = 4,    /* workspace smaller than hdqt_*_workspace_bytes  */
+  HDQT_ERR_NONFINITE = 5,    /* (device) NaN/Inf in a transformed operand      */
+  HDQT_ERR_TIMEOUT = 6,      /* (device) a bounded wait inside a kernel ran out*/
+  HDQT_ERR_CUDA = 7          /* a CUDA runtime / driver call failed            */
+} hdqt_status_t;
+
+typedef enum {
+  HDQT_ROUND_NEAREST = 0,    /* ties to even                                   */
+  HDQT_ROUND_STOCHASTIC = 1  /* Philox4x32-10 stream keyed by (seed, tag, idx) */
+} hdqt_round_t;
+
+/* flags for the GEMM entry points */
+#define HDQT_FLAG_NO_MERGE 1u /* never merge provably clamp-free tiles (see hdqt_gemm_i8_tiled) */
+
+/*
+ * Parameters of one HDQT GEMM Out[M,N] = A[M,K] B[K,N] (Section 3).
+ * Defaults of the paper: in_bits 4, acc_bits 8, acc_tile 32, had_block 32,
+ * acc_shift 0; clip 0.975 forward, 1.0 backward (Section 4).
+ */
+typedef struct hdqt_gemm_desc {
+  int32_t in_bits;    /* b   : 2..8, bit width of the operand codes                    */
+  int32_t acc_bits;   /* b_a : 2..32, bit width of a tile accumulator; 32 = unquantised */
+  int32_t acc_tile;   /* s   : tile length along K, a multiple of 32; 0 = whole K      */
+  int32_t acc_shift;  /* r   : tile sums are divided by 2^r (round-half-even) before the
+                               clamp to b_a bits; 0 = plain saturating accumulator      */
+  int32_t had_block;  /* n_h : Hadamard block, power of two in 1..32; 1 = no transform  */
+  float clip_a;       /* rho : operand A is scaled so that rho*max|x| maps to 2^(b-1)   */
+  float clip_b;
+  int32_t round_a;    /* hdqt_round_t for operand A                                    */
+  int32_t round_b;
+  uint64_t seed;      /* Philox key                                                    */
+  uint32_t tag_a;     /* Philox stream tag per operand: counter word 2                 */
+  uint32_t tag_b;
+  const float* amax_a; /* optional device scalar: max|H-domain A| supplied by the caller
+                          (skips the calibration pass); NULL = measure                 */
+  const float* amax_b;
+  uint32_t flags;     /* HDQT_FLAG_*                                                   */
+} hdqt_gemm_desc_t;
+
+/* Fills *d with the paper's defaults for kind 0 = forward, 1 = dgrad, 2 = wgrad
+ * (rounding modes and clip per Section 3 / Section 4). `d` is a host pointer. */
+void hdqt_default_desc(hdqt_gemm_desc_t* d, int kind);
+
+/* K rounded up to whole Hadamard blocks and 32-wide tiles (zero padding leaves
+ * X W unchanged; Section 3 defines H only for whole blocks). */
+int64_t hdqt_padded_k(int64_t K, int32_t had_block);
+
+const char* hdqt_status_string(hdqt_status_t s);
+
+/* ------------------------------------------------------------------------ */
+/* Transform + quantize (Section 3: Hadamard paragraph and definition of Q)   */
+/* ------------------------------------------------------------------------ */
+
+/*
+ * amax_out[0] = max |x H| over the zero-padded tensor, x H being the block-
+ * diagonal transform of `src` along K (the calibration maximum of Section 3).
+ *
+ * src: fp32, logical shape [rows, K]; element (r, k) is src[r*ld_row + k*ld_k].
+ *      Exactly one of ld_row, ld_k must be 1 (K contiguous, or K strided with
+ *      the row index contiguous); the other must be a multiple of 4.
+ * Non-finite values set HDQT_ERR_NONFINITE in *dev_status.
+ */
+hdqt_status_t hdqt_absmax_hadamard(const float* src, int64_t rows, int64_t K,
+                                   int64_t ld_row, int64_t ld_k, int32_t had_block,
+                                   float* amax_out, int32_t* dev_status, void* stream);
+
+/*
+ * codes[rows, K_pad] = Q(src H) with `bits`-bit two's-complement codes in int8
+ * lanes; step_out[0] = value of one code unit (codes*step ~ src H).
+ *
+ *   t = clip*amax, v = (src H) * (2^(bits-1) / t)
+ *   nearest   : code = clamp(rint(v))
+ *   stochastic: code = clamp(floor((rint(v*2^16) + u16) / 2^16)), u16 = 16 bits of
+ *               Philox4x32-10(counter = (g lo, g hi, tag, 0), key = seed), g = idx/8,
+ *               idx = r*K_pad + k; element idx%8 takes half (idx&1) of word (idx%8)/2
+ *   clamp to [-2^(bits-1), 2^(bits-1)-1]; all-zero tensor -> zero codes, step 0.
+ *
+ * amax_in : optional device scalar max|src H|; NULL = measure it first (one more
+ *           read pass over src) into the workspace.
+ * tile_norms: optional int32 [ceil(rows/128), K_pad/32]: for every block of 128
+ *           rows and every 32-wide K tile, max over the rows of sum(code^2); lets
+ *           the GEMM prove that a tile cannot clamp.  NULL = not produced.
+ * workspace: at least hdqt_quantize_workspace_bytes(rows, K, had_block) bytes (holds the
+ *           measured maximum and per-row tile norms).
+ */
+hdqt_status_t hdqt_quantize_hadamard(const float* src, int64_t rows, int64_t K,
+                                     int64_t ld_row, int64_t ld_k, int32_t had_block,
+                                     int32_t bits, float clip, int32_t mode,
+                                     uint64_t seed, uint32_t tag, const float* amax_in,
+                                     int8_t* codes, float* step_out, int32_t* tile_norms,
+                                     void* workspace, size_t workspace_bytes,
+                                     int32_t* dev_status, void* stream);
+
+size_t hdqt_quantize_workspace_bytes(int64_t rows, int64_t K, int32_t had_block);
+
+/* ------------------------------------------------------------------------ */
+/* Tiled integer GEMM with low-bit tile accumulators (Section 3, last para.)  */
+/* ------------------------------------------------------------------------ */
+
+/*
+ * out[m, n] = fp32(S[m, n]) * fp32(step_a*step_b*2^r / had_block),
+ *   S = sum over tiles t of clamp(rne(P_t / 2^r), -2^(b_a-1), 2^(b_a-1)-1),
+ *   P_t[m, n] = sum over the tile's k of Aq[m, k]*Bq[n, k]          (exact).
+ *
+ * Aq [M, K_pad], Bq [N, K_pad]: int8 codes, K contiguous, K_pad % 32 == 0,
+ *     |code| <= 2^(bits-1) with bits <= 8.
+ * step_a, step_b: device scalars written by hdqt_quantize_hadamard.
+ * out   : fp32 [M, ld_out] row-major, ld_out >= N.
+ * S_out : optional int32 [M, N] (dense): the integer sums S.
+ * tiles_out: optional int8/int16 debug output, see `tiles_elem_bytes`: [T, M, N]
+ *     per-tile accumulator contents c_t; forces every tile through the clamp path.
+ * tiles_elem_bytes: 1 (acc_bits <= 8) or 2 (acc_bits <= 16); ignored if tiles_out NULL.
+ * norms_a [ceil(M/128), K_pad/32], norms_b [ceil(N/128), K_pad/32]: optional
+ *     tile_norms from the quantizer.  When both are given, acc_shift == 0 and
+ *     HDQT_FLAG_NO_MERGE is clear, consecutive tiles for which the Cauchy-Schwarz
+ *     bound proves |P_t| <= 2^(b_a-1)-1 for a whole 128x256 output block are
+ *     accumulated together on the tensor core; the clamp is the identity on such
+ *     tiles, so the result is bit-identical to the tile-by-tile path.
+ * workspace: at least hdqt_gemm_i8_workspace_bytes(M, N, K_pad) bytes.
+ */
+hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, const float* step_a,
+                                 const float* step_b, int64_t M, int64_t N, int64_t K_pad,
+                                 int32_t acc_bits, int32_t acc_tile, int32_t acc_shift,
+                                 int32_t had_block, float* out, int64_t ld_out,
+                                 int32_t* S_out, void* tiles_out, int32_t tiles_elem_bytes,
+                                 const int32_t* norms_a, const int32_t* norms_b,
+                                 uint32_t flags, void* workspace, size_t workspace_bytes,
+                                 int32_t* dev_status, void* stream);
+
+size_t hdqt_gemm_i8_workspace_bytes(int64_t M, int64_t N, int64_t K_pad);
+
+/*
+ * shift_out[0] (device int32) = smallest r >= 0 for which no tile of the given
+ * operands clamps: max calibration (Section 3) of the accumulator restricted to
+ * powers of two.  Operand layout as in hdqt_gemm_i8_tiled.
+ */
+hdqt_status_t hdqt_calibrate_acc_shift(const int8_t* Aq, const int8_t* Bq, int64_t M,
+                                       int64_t N, int64_t K_pad, int32_t acc_bits,
+                                       int32_t acc_tile, int32_t* shift_out,
+                                       void* workspace, size_t workspace_bytes,
+                                       int32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------ */
+/* The three training GEMMs of one linear layer (Section 3: Z = X W and the    */
+/* backward products; X [Nb, D] activations, W weights, G = dL/dY [Nb, C])     */
+/* ------------------------------------------------------------------------ */
+
+/* W storage: w_is_cd == 0: W[D, C] row-major (the paper's W in R^{DxC});
+ *            w_is_cd != 0: W[C, D] row-major (the transposed, "linear layer" layout). */
+
+/* Y[Nb, C] = X[Nb, D] W : contraction over D. */
+hdqt_status_t hdqt_gemm_fwd(const hdqt_gemm_desc_t* desc /*host*/, const float* X,
+                            const float* W, float* Y, int64_t Nb, int64_t D, int64_t C,
+                            int32_t w_is_cd, void* workspace, size_t workspace_bytes,
+                            int32_t* dev_status, void* stream);
+
+/* dX[Nb, D] = G[Nb, C] W^T : contraction over C. */
+hdqt_status_t hdqt_gemm_dgrad(const hdqt_gemm_desc_t* desc /*host*/, const float* G,
+                              const float* W, float* dX, int64_t Nb, int64_t D, int64_t C,
+                              int32_t w_is_cd, void* workspace, size_t workspace_bytes,
+                              int32_t* dev_status, void* stream);
+
+/* dW = X^T G : contraction over the batch Nb; dW is written in W's layout
+ * ([D, C] or, if w_is_cd, [C, D]). */
+hdqt_status_t hdqt_gemm_wgrad(const hdqt_gemm_desc_t* desc /*host*/, const float* X,
+                              const float* G, float* dW, int64_t Nb, int64_t D, int64_t C,
+                              int32_t w_is_cd, void* workspace, size_t workspace_bytes,
+                              int32_t* dev_status, void* stream);
+
+/* Workspace for any of the three calls on a GEMM of the given size
+ * (codes of both operands, scales, tile norms, GEMM scratch). */
+size_t hdqt_workspace_bytes(const hdqt_gemm_desc_t* desc /*host*/, int64_t M, int64_t N,
+                            int64_t K);
+
+/*
+ * Host-side view of the workspace layout used by the three calls above, so a
+ * test harness can read the intermediate codes and scales back after a call.
+ * All offsets are in bytes from `workspace`.
+ */
+typedef struct hdqt_ws_layout {
+  size_t codes_a, codes_b;   /* int8 [M, K_pad], [N, K_pad]          */
+  size_t step_a, step_b;     /* fp32 scalars                         */
+  size_t amax_a, amax_b;     /* fp32 scalars                         */
+  size_t norms_a, norms_b;   /* int32 tile norms                     */
+  size_t gemm_ws;            /* scratch of hdqt_gemm_i8_tiled        */
+  size_t total;
+  int64_t k_pad;
+} hdqt_ws_layout_t;
+
+hdqt_status_t hdqt_workspace_layout(const hdqt_gemm_desc_t* desc /*host*/, int64_t M,
+                                    int64_t N, int64_t K, hdqt_ws_layout_t* out /*host*/);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HDQT_H_ */

@@ -1,0 +1,74 @@
+// Shared declarations of the HDQT CUDA library (device helpers + internal launchers).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hdqt.h"
+
+namespace hdqt {
+
+constexpr int kNumSMsHint = 148;  // B200; grids are sized from the queried SM count at run time
+
+// Sticky maximum into the caller's device status word (may be null).
+__device__ __forceinline__ void report_status(int32_t* dev_status, int32_t code) {
+  if (dev_status != nullptr) atomicMax(dev_status, code);
+}
+
+// ---- Philox4x32-10 (Salmon et al., SC'11): counter-based generator for stochastic rounding ----
+struct Philox4 {
+  uint32_t w[4];
+};
+
+__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += W0;
+    k1 += W1;
+  }
+  Philox4 o;
+  o.w[0] = c0; o.w[1] = c1; o.w[2] = c2; o.w[3] = c3;
+  return o;
+}
+
+// Parameters of the quantizer derived from the calibration maximum (all fp32, one rounding each).
+struct QuantScale {
+  float m;     // 2^(bits-1) / (clip*amax): multiplier from H-domain value to code units
+  float step;  // clip*amax*2^-(bits-1): value of one code unit
+  bool zero;   // amax == 0 (all codes are 0)
+  bool bad;    // amax or m not finite
+};
+
+__device__ __forceinline__ QuantScale make_quant_scale(float amax, float clip, int bits) {
+  QuantScale q;
+  const float half_range = (float)(1 << (bits - 1));
+  const float t = __fmul_rn(clip, amax);
+  q.m = __fdiv_rn(half_range, t);
+  q.step = __fmul_rn(t, __fdiv_rn(1.0f, half_range));
+  q.zero = (amax == 0.0f);
+  q.bad = !(isfinite(amax)) || (!q.zero && !isfinite(q.m));
+  if (q.zero || q.bad) { q.m = 0.0f; q.step = 0.0f; }
+  return q;
+}
+
+// ---- internal launchers (defined in the .cu files) ----
+hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
+                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s);
+
+hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
+                              int32_t had_block, int32_t bits, float clip, int32_t mode, uint64_t seed,
+                              uint32_t tag, const float* amax, int8_t* codes, float* step_out,
+                              int32_t* tile_norms, uint16_t* row_norms_scratch, int32_t* dev_status,
+                              cudaStream_t s);
+
+int sm_count();
+
+}  // namespace hdqt

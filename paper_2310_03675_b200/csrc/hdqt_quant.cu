@@ -1,0 +1,448 @@
+// FWHT + calibration maximum + quantizer kernels (paper Section 3: Hadamard paragraph,
+// definition of Q, stochastic rounding; Section 4: clip factor).
+//
+// Two memory layouts of the source operand are served:
+//   * K contiguous ("kc"): a thread owns 8 consecutive k of one row; a 32-wide Hadamard
+//     block is spread over 4 neighbouring lanes: strides 1,2,4 run in registers, strides 8,16
+//     through warp shuffles.  Loads are 2 x 128-bit per thread, stores 64-bit per thread.
+//   * K strided ("ks", the row index is contiguous): a thread owns one whole 32-wide block of
+//     one row; a warp reads 32 consecutive rows per load instruction (128 bytes, coalesced),
+//     all five butterfly stages run in registers, and the thread writes its 32 codes as one
+//     32-byte segment of the K-contiguous code row (a fused transpose).
+//
+// Both are HBM-bound streaming kernels: 4 B/element read (+1 B/element written when
+// quantizing).  Butterfly order is ascending stride, every add/sub is a single fp32 rounding,
+// so the transformed values - and hence the codes - are bit-identical for both layouts.
+#include "hdqt_common.cuh"
+
+namespace hdqt {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+// ---- butterflies ------------------------------------------------------------------------
+
+// strides 1, 2, 4 on 8 register values (only those below had_block)
+__device__ __forceinline__ void fwht8_regs(float (&x)[8], int had_block) {
+  if (had_block > 1) {
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+      const float a = x[i], b = x[i + 1];
+      x[i] = __fadd_rn(a, b);
+      x[i + 1] = __fsub_rn(a, b);
+    }
+  }
+  if (had_block > 2) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if ((i & 2) == 0) {
+        const float a = x[i], b = x[i + 2];
+        x[i] = __fadd_rn(a, b);
+        x[i + 2] = __fsub_rn(a, b);
+      }
+    }
+  }
+  if (had_block > 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float a = x[i], b = x[i + 4];
+      x[i] = __fadd_rn(a, b);
+      x[i + 4] = __fsub_rn(a, b);
+    }
+  }
+}
+
+// strides 8 and 16 across lanes (lane^1, lane^2); the whole warp must call this
+__device__ __forceinline__ void fwht8_lanes(float (&x)[8], int had_block, int lane) {
+  if (had_block > 8) {
+    const bool upper = lane & 1;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float y = __shfl_xor_sync(0xFFFFFFFFu, x[i], 1);
+      x[i] = upper ? __fsub_rn(y, x[i]) : __fadd_rn(x[i], y);
+    }
+  }
+  if (had_block > 16) {
+    const bool upper = lane & 2;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float y = __shfl_xor_sync(0xFFFFFFFFu, x[i], 2);
+      x[i] = upper ? __fsub_rn(y, x[i]) : __fadd_rn(x[i], y);
+    }
+  }
+}
+
+// all stages on 32 register values
+__device__ __forceinline__ void fwht32_regs(float (&x)[32], int had_block) {
+#pragma unroll
+  for (int h = 1; h < 32; h <<= 1) {
+    if (h < had_block) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        if ((i & h) == 0) {
+          const float a = x[i], b = x[i + h];
+          x[i] = __fadd_rn(a, b);
+          x[i + h] = __fsub_rn(a, b);
+        }
+      }
+    }
+  }
+}
+
+// ---- loads ------------------------------------------------------------------------------
+
+// 8 consecutive k of one row, zero beyond K. `vec` = row base and stride are 16-byte aligned.
+__device__ __forceinline__ void load8_kc(const float* __restrict__ row, int64_t k0, int64_t K, bool vec,
+                                         float (&x)[8]) {
+  if (vec && k0 + 8 <= K) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(row + k0));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(row + k0 + 4));
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = (k0 + i < K) ? __ldg(row + k0 + i) : 0.0f;
+  }
+}
+
+// ---- quantizer --------------------------------------------------------------------------
+
+struct QuantParams {
+  float m;
+  int lo, hi;
+  int mode;          // hdqt_round_t
+  bool sr_magic;     // |v| < 64 guaranteed: fixed-point conversion through the fp32 adder
+  uint32_t k0, k1, tag;
+};
+
+// codes of 8 consecutive elements; `g` = (linear index of the first element) / 8
+__device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams& p, uint64_t g,
+                                          int (&c)[8]) {
+  if (p.mode == HDQT_ROUND_NEAREST) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float v = __fmul_rn(x[i], p.m);
+      // rint through the fp32 adder: exact for |v| < 2^22
+      const int q = __float_as_int(__fadd_rn(v, 12582912.0f)) - 0x4B400000;
+      c[i] = min(max(q, p.lo), p.hi);
+    }
+  } else {
+    const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, 0u, p.k0, p.k1);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float v = __fmul_rn(x[i], p.m);
+      const uint32_t word = rnd.w[i >> 1];
+      const int u16 = (i & 1) ? (int)(word >> 16) : (int)(word & 0xFFFFu);
+      int v_fx;  // rint(v * 2^16), a Q.16 fixed-point integer
+      if (p.sr_magic) {
+        // for v in [-64, 64): v + 192 lies in [128, 256) where one ulp is 2^-16
+        v_fx = __float_as_int(__fadd_rn(v, 192.0f)) - 0x43400000;
+      } else {
+        v_fx = __float2int_rn(__fmul_rn(v, 65536.0f));
+      }
+      const int q = (v_fx + u16) >> 16;  // floor((v_fx + u16) / 2^16)
+      c[i] = min(max(q, p.lo), p.hi);
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
+  return (uint32_t)(a & 0xFF) | ((uint32_t)(b & 0xFF) << 8) | ((uint32_t)(c & 0xFF) << 16) |
+         ((uint32_t)(d & 0xFF) << 24);
+}
+
+__device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bits, float clip, int mode,
+                                                   uint64_t seed, uint32_t tag) {
+  QuantParams p;
+  p.m = qs.m;
+  p.lo = -(1 << (bits - 1));
+  p.hi = (1 << (bits - 1)) - 1;
+  p.mode = mode;
+  p.sr_magic = ((float)(1 << (bits - 1)) <= 32.0f * clip);  // |v| <= 32 (1 + eps)
+  p.k0 = (uint32_t)seed;
+  p.k1 = (uint32_t)(seed >> 32);
+  p.tag = tag;
+  return p;
+}
+
+// ---- block-wide max -----------------------------------------------------------------------
+
+__device__ __forceinline__ void block_absmax_commit(uint32_t mx, float* amax_out, int32_t* dev_status) {
+  __shared__ uint32_t smax[kThreads / 32];
+  mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) smax[warp] = mx;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t v = (lane < kThreads / 32) ? smax[lane] : 0u;
+    v = __reduce_max_sync(0xFFFFFFFFu, v);
+    if (lane == 0) {
+      // non-negative floats order like their bit patterns
+      atomicMax(reinterpret_cast<uint32_t*>(amax_out), v);
+      if (v >= 0x7F800000u) report_status(dev_status, HDQT_ERR_NONFINITE);
+    }
+  }
+}
+
+// ---- K-contiguous kernels -------------------------------------------------------------------
+
+__global__ void __launch_bounds__(kThreads)
+absmax_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_row, int64_t K_pad,
+                 int had_block, bool vec, float* amax_out, int32_t* dev_status) {
+  const int64_t chunks_per_row = K_pad >> 3;
+  const int64_t total = rows * chunks_per_row;
+  const int64_t total_warp = (total + 31) & ~int64_t(31);
+  const int lane = threadIdx.x & 31;
+  uint32_t mx = 0u;
+  for (int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x; c < total_warp;
+       c += (int64_t)gridDim.x * kThreads) {
+    float x[8];
+    if (c < total) {
+      const int64_t r = c / chunks_per_row;
+      const int64_t k0 = (c - r * chunks_per_row) << 3;
+      load8_kc(src + r * ld_row, k0, K, vec, x);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[i] = 0.0f;
+    }
+    fwht8_regs(x, had_block);
+    fwht8_lanes(x, had_block, lane);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) mx = max(mx, abs_bits(x[i]));
+  }
+  block_absmax_commit(mx, amax_out, dev_status);
+}
+
+__global__ void __launch_bounds__(kThreads)
+quantize_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_row, int64_t K_pad,
+                   int had_block, bool vec, int bits, float clip, int mode, uint64_t seed, uint32_t tag,
+                   const float* __restrict__ amax_ptr, int8_t* __restrict__ codes, float* step_out,
+                   uint16_t* __restrict__ row_norms, int32_t* dev_status) {
+  const QuantScale qs = make_quant_scale(__ldg(amax_ptr), clip, bits);
+  const QuantParams p = make_params(qs, bits, clip, mode, seed, tag);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *step_out = qs.step;
+    if (qs.bad) report_status(dev_status, HDQT_ERR_NONFINITE);
+  }
+  const int64_t chunks_per_row = K_pad >> 3;
+  const int64_t total = rows * chunks_per_row;
+  const int64_t total_warp = (total + 31) & ~int64_t(31);
+  const int lane = threadIdx.x & 31;
+  for (int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x; c < total_warp;
+       c += (int64_t)gridDim.x * kThreads) {
+    float x[8];
+    const bool valid = c < total;
+    int64_t r = 0, k0 = 0;
+    if (valid) {
+      r = c / chunks_per_row;
+      k0 = (c - r * chunks_per_row) << 3;
+      load8_kc(src + r * ld_row, k0, K, vec, x);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[i] = 0.0f;
+    }
+    fwht8_regs(x, had_block);
+    fwht8_lanes(x, had_block, lane);
+    int q[8];
+    quantize8(x, p, (uint64_t)c, q);  // linear index of the chunk's first element is 8*c
+    if (row_norms != nullptr) {
+      int ss = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ss += q[i] * q[i];
+      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+      if (valid && (lane & 3) == 0) row_norms[r * (K_pad >> 5) + (k0 >> 5)] = (uint16_t)ss;
+    }
+    if (valid) {
+      uint2 out;
+      out.x = pack4(q[0], q[1], q[2], q[3]);
+      out.y = pack4(q[4], q[5], q[6], q[7]);
+      *reinterpret_cast<uint2*>(codes + r * K_pad + k0) = out;
+    }
+  }
+}
+
+// max over each block of 128 rows of the per-row tile norms
+__global__ void block_norms_kernel(const uint16_t* __restrict__ row_norms, int64_t rows, int64_t T,
+                                   int32_t* __restrict__ tile_norms) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t rb = blockIdx.y;
+  if (t >= T) return;
+  const int64_t r0 = rb * 128, r1 = min(rows, r0 + 128);
+  int mx = 0;
+  for (int64_t r = r0; r < r1; ++r) mx = max(mx, (int)row_norms[r * T + t]);
+  tile_norms[rb * T + t] = mx;
+}
+
+// ---- K-strided kernels ------------------------------------------------------------------------
+// element (r, k) = src[k*ld_k + r]; thread = (row r, 32-block kb); r is the fast thread index.
+
+__device__ __forceinline__ void load32_ks(const float* __restrict__ src, int64_t r, int64_t kb, int64_t K,
+                                          int64_t ld_k, float (&x)[32]) {
+  const float* p = src + (kb << 5) * ld_k + r;
+  const int64_t k_left = K - (kb << 5);
+  if (k_left >= 32) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) x[i] = __ldg(p + i * ld_k);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) x[i] = (i < k_left) ? __ldg(p + i * ld_k) : 0.0f;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+absmax_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_k, int64_t K_pad,
+                 int had_block, float* amax_out, int32_t* dev_status) {
+  const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
+  const int64_t total = rows_pad * (K_pad >> 5);
+  uint32_t mx = 0u;
+  for (int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x; id < total;
+       id += (int64_t)gridDim.x * kThreads) {
+    const int64_t kb = id / rows_pad;
+    const int64_t r = id - kb * rows_pad;
+    if (r < rows) {
+      float x[32];
+      load32_ks(src, r, kb, K, ld_k, x);
+      fwht32_regs(x, had_block);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) mx = max(mx, abs_bits(x[i]));
+    }
+  }
+  block_absmax_commit(mx, amax_out, dev_status);
+}
+
+__global__ void __launch_bounds__(kThreads)
+quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_k, int64_t K_pad,
+                   int had_block, int bits, float clip, int mode, uint64_t seed, uint32_t tag,
+                   const float* __restrict__ amax_ptr, int8_t* __restrict__ codes, float* step_out,
+                   int32_t* __restrict__ tile_norms, int32_t* dev_status) {
+  __shared__ int s_norm[kThreads / 32];
+  const QuantScale qs = make_quant_scale(__ldg(amax_ptr), clip, bits);
+  const QuantParams p = make_params(qs, bits, clip, mode, seed, tag);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *step_out = qs.step;
+    if (qs.bad) report_status(dev_status, HDQT_ERR_NONFINITE);
+  }
+  // rows are padded to a multiple of the block size so that one thread block never straddles
+  // two 32-blocks of K and always covers whole 128-row groups (needed for the tile norms)
+  const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
+  const int64_t T = K_pad >> 5;
+  const int64_t total = rows_pad * T;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int64_t id0 = (int64_t)blockIdx.x * kThreads; id0 < total; id0 += (int64_t)gridDim.x * kThreads) {
+    const int64_t id = id0 + threadIdx.x;
+    const int64_t kb = id0 / rows_pad;          // uniform over the block
+    const int64_t r = id - kb * rows_pad;
+    int ss = 0;
+    if (r < rows) {
+      float x[32];
+      load32_ks(src, r, kb, K, ld_k, x);
+      fwht32_regs(x, had_block);
+      uint32_t w[8];
+      const uint64_t g0 = (uint64_t)(r * K_pad + (kb << 5)) >> 3;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float x8[8];
+        int q[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x8[i] = x[8 * j + i];
+        quantize8(x8, p, g0 + j, q);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ss += q[i] * q[i];
+        w[2 * j] = pack4(q[0], q[1], q[2], q[3]);
+        w[2 * j + 1] = pack4(q[4], q[5], q[6], q[7]);
+      }
+      uint4* dst = reinterpret_cast<uint4*>(codes + r * K_pad + (kb << 5));
+      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+    if (tile_norms != nullptr) {  // uniform branch
+      ss = __reduce_max_sync(0xFFFFFFFFu, ss);
+      __syncthreads();
+      if (lane == 0) s_norm[warp] = ss;
+      __syncthreads();
+      if (threadIdx.x < kThreads / 128) {
+        const int64_t r_base = (id0 - kb * rows_pad) + threadIdx.x * 128;
+        if (r_base < rows) {
+          int mx = 0;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mx = max(mx, s_norm[threadIdx.x * 4 + i]);
+          tile_norms[(r_base >> 7) * T + kb] = mx;
+        }
+      }
+    }
+  }
+}
+
+int g_sm_count = 0;
+
+}  // namespace
+
+int sm_count() {
+  if (g_sm_count == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      n = kNumSMsHint;
+    }
+    g_sm_count = n;
+  }
+  return g_sm_count;
+}
+
+static int grid_for(int64_t work_items, int per_block, int blocks_per_sm) {
+  const int64_t need = (work_items + per_block - 1) / per_block;
+  const int64_t cap = (int64_t)sm_count() * blocks_per_sm;
+  return (int)(need < 1 ? 1 : (need < cap ? need : cap));
+}
+
+hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
+                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s) {
+  const int64_t K_pad = hdqt_padded_k(K, had_block);
+  if (cudaMemsetAsync(amax_out, 0, sizeof(float), s) != cudaSuccess) return HDQT_ERR_CUDA;
+  if (ld_k == 1) {
+    const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
+    const int64_t total = rows * (K_pad >> 3);
+    absmax_kc_kernel<<<grid_for(total, kThreads, 8), kThreads, 0, s>>>(src, rows, K, ld_row, K_pad, had_block,
+                                                                     vec, amax_out, dev_status);
+  } else {
+    const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
+    const int64_t total = rows_pad * (K_pad >> 5);
+    absmax_ks_kernel<<<grid_for(total, kThreads, 4), kThreads, 0, s>>>(src, rows, K, ld_k, K_pad, had_block,
+                                                                     amax_out, dev_status);
+  }
+  return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
+}
+
+hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
+                              int32_t had_block, int32_t bits, float clip, int32_t mode, uint64_t seed,
+                              uint32_t tag, const float* amax, int8_t* codes, float* step_out,
+                              int32_t* tile_norms, uint16_t* row_norms_scratch, int32_t* dev_status,
+                              cudaStream_t s) {
+  const int64_t K_pad = hdqt_padded_k(K, had_block);
+  const int64_t T = K_pad >> 5;
+  if (ld_k == 1) {
+    const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
+    const int64_t total = rows * (K_pad >> 3);
+    uint16_t* rn = tile_norms ? row_norms_scratch : nullptr;
+    quantize_kc_kernel<<<grid_for(total, kThreads, 8), kThreads, 0, s>>>(
+        src, rows, K, ld_row, K_pad, had_block, vec, bits, clip, mode, seed, tag, amax, codes, step_out, rn,
+        dev_status);
+    if (tile_norms) {
+      dim3 grid((unsigned)((T + 127) / 128), (unsigned)((rows + 127) / 128));
+      block_norms_kernel<<<grid, 128, 0, s>>>(rn, rows, T, tile_norms);
+    }
+  } else {
+    const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
+    const int64_t total = rows_pad * T;
+    quantize_ks_kernel<<<grid_for(total, kThreads, 4), kThreads, 0, s>>>(
+        src, rows, K, ld_k, K_pad, had_block, bits, clip, mode, seed, tag, amax, codes, step_out, tile_norms,
+        dev_status);
+  }
+  return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
+}
+
+}  // namespace hdqt

@@ -1,0 +1,227 @@
+"""GPU parity: tiled integer GEMM and the three training GEMMs against the CPU oracle.
+Integers (codes, per-tile accumulators, sums) bit-exact; fp32 outputs within 1e-5 relative."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hdqt_oracle as O
+from paper_2310_03675_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 1e-5   # fp32 output tolerance stated for this path (in practice the outputs are identical)
+
+
+@pytest.fixture(scope="module")
+def hdqt():
+    from paper_2310_03675_b200 import hdqt as mod
+    return mod
+
+
+def _dev(x):
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def _assert_close(got, want):
+    got = got.astype(np.float64)
+    want = want.astype(np.float64)
+    denom = max(np.abs(want).max(), 1e-30)
+    assert np.abs(got - want).max() / denom <= REL_TOL
+
+
+def _codes(rng, rows, K, lo=-8, hi=8):
+    return rng.integers(lo, hi, size=(rows, K)).astype(np.int8)
+
+
+GEMM_SHAPES = [(32, 64, 128), (1, 1, 32), (128, 256, 32), (129, 257, 160), (300, 520, 416), (64, 12, 256), (260, 100, 96)]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+def test_i8_tiled_default_parameters(hdqt, M, N, K):
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    Aq, Bq = _codes(rng, M, K), _codes(rng, N, K)
+    sa, sb = np.float32(0.0123), np.float32(3.5e-4)
+    want_out, want_S, want_tiles = O.gemm_i8_tiled(Aq, Bq, sa, sb, 8, 32, 0, 32, want_tiles=True)
+    status = hdqt.new_status("cuda")
+    out, S, tiles = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), torch.tensor([sa], device="cuda"),
+                                       torch.tensor([sb], device="cuda"), want_S=True, want_tiles=True,
+                                       dev_status=status)
+    hdqt.check_device_status(status)
+    assert np.array_equal(tiles.cpu().numpy().astype(np.int64), want_tiles)
+    assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
+    _assert_close(out.cpu().numpy(), want_out)
+    # and without the debug output (the production kernel variant)
+    out2, S2, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), torch.tensor([sa], device="cuda"),
+                                     torch.tensor([sb], device="cuda"), want_S=True, dev_status=status)
+    hdqt.check_device_status(status)
+    assert np.array_equal(S2.cpu().numpy().astype(np.int64), want_S)
+    assert np.array_equal(out2.cpu().numpy(), out.cpu().numpy())
+
+
+@pytest.mark.parametrize("acc_bits,acc_tile,acc_shift", [(8, 32, 2), (8, 32, 4), (4, 32, 0), (6, 32, 3), (12, 32, 0),
+                                                         (16, 64, 0), (8, 64, 1), (8, 128, 3), (8, 0, 0), (32, 0, 0),
+                                                         (32, 32, 0), (8, 96, 0)])
+def test_i8_tiled_parameter_family(hdqt, acc_bits, acc_tile, acc_shift):
+    rng = np.random.default_rng(acc_bits * 100 + acc_tile + acc_shift)
+    M, N, K = 140, 270, 448
+    Aq, Bq = _codes(rng, M, K), _codes(rng, N, K)
+    sa, sb = np.float32(0.5), np.float32(0.25)
+    want_tiles_flag = acc_bits <= 16
+    want_out, want_S, want_tiles = O.gemm_i8_tiled(Aq, Bq, sa, sb, acc_bits, acc_tile, acc_shift, 32,
+                                                   want_tiles=want_tiles_flag)
+    status = hdqt.new_status("cuda")
+    out, S, tiles = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), torch.tensor([sa], device="cuda"),
+                                       torch.tensor([sb], device="cuda"), acc_bits, acc_tile, acc_shift, 32,
+                                       want_S=True, want_tiles=want_tiles_flag, dev_status=status)
+    hdqt.check_device_status(status)
+    if want_tiles_flag:
+        assert np.array_equal(tiles.cpu().numpy().astype(np.int64), want_tiles)
+    assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
+    _assert_close(out.cpu().numpy(), want_out)
+
+
+def test_i8_tiled_saturating_and_8bit_codes(hdqt):
+    """All-7 codes clamp every tile at 127; full-range int8 codes exercise the signed 8-bit MMA path."""
+    A = np.full((130, 96), 7, np.int8)
+    B = np.full((20, 96), 7, np.int8)
+    one = torch.ones(1, device="cuda")
+    _, S, _ = hdqt.gemm_i8_tiled(_dev(A), _dev(B), one, one, want_S=True)
+    assert (S == 3 * 127).all().item()
+    _, S, _ = hdqt.gemm_i8_tiled(_dev(-A - 1), _dev(B), one, one, want_S=True)      # -8 * 7 * 32 -> -128
+    assert (S == 3 * -128).all().item()
+    rng = np.random.default_rng(3)
+    A8, B8 = _codes(rng, 64, 128, -128, 128), _codes(rng, 48, 128, -128, 128)
+    _, want_S, _ = O.gemm_i8_tiled(A8, B8, 1.0, 1.0, 32, 0, 0, 32)
+    _, S, _ = hdqt.gemm_i8_tiled(_dev(A8), _dev(B8), one, one, 32, 0, 0, 32, want_S=True)
+    assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
+
+
+def test_i8_tiled_strided_output_and_canaries(hdqt):
+    rng = np.random.default_rng(5)
+    M, N, K = 70, 33, 64
+    Aq, Bq = _codes(rng, M, K), _codes(rng, N, K)
+    want_out, _, _ = O.gemm_i8_tiled(Aq, Bq, 1.0, 1.0)
+    big = torch.full((M + 2, N + 7), -777.0, device="cuda")
+    view = big[1:M + 1, 3:3 + N]
+    one = torch.ones(1, device="cuda")
+    hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), one, one, out=view)
+    torch.cuda.synchronize()
+    assert np.array_equal(view.cpu().numpy(), want_out)
+    mask = torch.ones_like(big, dtype=torch.bool)
+    mask[1:M + 1, 3:3 + N] = False
+    assert (big[mask] == -777.0).all().item()
+
+
+def test_calibrate_acc_shift(hdqt):
+    rng = np.random.default_rng(6)
+    for lo, hi, bits in ((-8, 8, 8), (-2, 3, 8), (-8, 8, 6), (-8, 8, 12)):
+        Aq, Bq = _codes(rng, 40, 96, lo, hi), _codes(rng, 24, 96, lo, hi)
+        want = O.calibrate_acc_shift(Aq, Bq, bits, 32)
+        got = hdqt.calibrate_acc_shift(_dev(Aq), _dev(Bq), bits, 32).item()
+        assert got == want
+
+
+# ---- the three training GEMMs ----------------------------------------------------------------------
+
+def _run_three(hdqt, X, W, G, w_is_cd=False, **over):
+    """Runs fwd/dgrad/wgrad on the GPU and through the oracle; compares every intermediate."""
+    Xd, Gd = _dev(X), _dev(G)
+    Wd = _dev(W.T) if w_is_cd else _dev(W)
+    status = hdqt.new_status("cuda")
+    cases = [
+        ("fwd", hdqt.gemm_fwd, (Xd, Wd), O.gemm_fwd(X, W, O.fwd_desc(tag_a=0, tag_b=1, **over)), False),
+        ("dgrad", hdqt.gemm_dgrad, (Gd, Wd), O.gemm_dgrad(G, W, O.dgrad_desc(tag_a=2, tag_b=3, **over)), False),
+        ("wgrad", hdqt.gemm_wgrad, (Xd, Gd), O.gemm_wgrad(X, G, O.wgrad_desc(tag_a=4, tag_b=5, **over)), True),
+    ]
+    for kind, fn, args, want, is_wgrad in cases:
+        desc = hdqt.default_desc(kind, **over)
+        out, ws = fn(*args, desc=desc, w_is_cd=w_is_cd, dev_status=status)
+        hdqt.check_device_status(status, kind)
+        swapped = is_wgrad and w_is_cd
+        got_a, got_b = ws.codes_a().cpu().numpy(), ws.codes_b().cpu().numpy()
+        sa, sb = ws.scalar("step_a").item(), ws.scalar("step_b").item()
+        if swapped:
+            got_a, got_b, sa, sb = got_b, got_a, sb, sa
+        assert np.array_equal(got_a, want["Aq"]), kind
+        assert np.array_equal(got_b, want["Bq"]), kind
+        assert sa == float(want["step_a"]) and sb == float(want["step_b"]), kind
+        want_out = want["out"].T if swapped else want["out"]
+        _assert_close(out.cpu().numpy(), want_out)
+        # integer sums: re-run the integer GEMM on the codes the library produced
+        _, S, tiles = hdqt.gemm_i8_tiled(ws.codes_a(), ws.codes_b(), ws.scalar("step_a"), ws.scalar("step_b"),
+                                         desc.acc_bits, desc.acc_tile, desc.acc_shift, desc.had_block,
+                                         want_S=True, want_tiles=desc.acc_bits <= 16)
+        want_S = want["S"].T if swapped else want["S"]
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), kind
+        if tiles is not None:
+            _, _, want_tiles = O.gemm_i8_tiled(want["Aq"], want["Bq"], 1, 1, desc.acc_bits, desc.acc_tile,
+                                               desc.acc_shift, desc.had_block, want_tiles=True)
+            if swapped:
+                want_tiles = want_tiles.transpose(0, 2, 1)
+            assert np.array_equal(tiles.cpu().numpy().astype(np.int64), want_tiles), kind
+
+
+@pytest.mark.parametrize("w_is_cd", [False, True])
+def test_single_linear_layer(hdqt, w_is_cd):
+    """X [32,128] ~ N(0,1), W [128,64] ~ N(0,0.05^2), G [32,64] ~ 1e-3 t(3); seed 0."""
+    X, W, G = inputs.single_layer(0)
+    _run_three(hdqt, X, W, G, w_is_cd=w_is_cd, seed=0)
+
+
+@pytest.mark.parametrize("Nb,D,C", [(256, 1152, 512), (256, 512, 256), (256, 256, 12), (128, 561, 561), (128, 27, 64),
+                                    (130, 100, 7)])
+def test_mlp_and_ragged_layers(hdqt, Nb, D, C):
+    X = np.maximum(inputs.activations(Nb, D, seed=D), 0)        # post-ReLU activations
+    W = inputs.weights(D, C, seed=C)
+    G = inputs.gradients(Nb, C, seed=Nb + C)
+    _run_three(hdqt, X, W, G, seed=42)
+
+
+@pytest.mark.parametrize("over", [dict(acc_bits=12), dict(acc_bits=4), dict(in_bits=3, acc_bits=6), dict(in_bits=8, acc_bits=16),
+                                  dict(acc_tile=0), dict(had_block=1), dict(acc_shift=2), dict(acc_tile=64, acc_shift=1)])
+def test_bit_width_family_and_paper_arrangement(hdqt, over):
+    X, W, G = inputs.single_layer(1, Nb=96, D=160, C=72)
+    _run_three(hdqt, X, W, G, seed=7, **over)
+
+
+def test_im2col_like_wgrad_long_contraction(hdqt):
+    """wgrad with a long batch contraction (many tiles) and a narrow output."""
+    X = np.maximum(inputs.activations(4096, 576, seed=11), 0)
+    G = inputs.gradients(4096, 64, seed=12)
+    W = inputs.weights(576, 64, seed=13)
+    _run_three(hdqt, X, W, G, seed=3)
+
+
+def test_runs_are_bitwise_reproducible(hdqt):
+    X, W, G = inputs.single_layer(2, Nb=200, D=300, C=150)
+    Xd, Gd = _dev(X), _dev(G)
+    a, _ = hdqt.gemm_wgrad(Xd, Gd)
+    b, _ = hdqt.gemm_wgrad(Xd, Gd)
+    assert torch.equal(a, b)
+    c, _ = hdqt.gemm_wgrad(Xd, Gd, desc=hdqt.default_desc("wgrad", seed=1))
+    assert not torch.equal(a, c)
+
+
+def test_sampled_parity_at_sweep_size(hdqt):
+    """4096^3 dgrad-layout GEMM on heavy-tailed operands: codes in full, integer sums on sampled rows/columns."""
+    M = N = K = 4096
+    A = inputs.heavy_tailed_torch(M, K, seed=100, device="cuda")
+    B = inputs.heavy_tailed_torch(N, K, seed=101, device="cuda")
+    desc = hdqt.default_desc("dgrad", seed=9)
+    status = hdqt.new_status("cuda")
+    out, ws = hdqt.gemm_dgrad(A, B, desc=desc, dev_status=status)
+    hdqt.check_device_status(status)
+    want_a, sa, _ = O.quantize_hadamard(A.cpu().numpy(), 32, 4, 1.0, 1, seed=9, tag=desc.tag_a)
+    want_b, sb, _ = O.quantize_hadamard(B.cpu().numpy(), 32, 4, 1.0, 0, seed=9, tag=desc.tag_b)
+    assert np.array_equal(ws.codes_a().cpu().numpy(), want_a)
+    assert np.array_equal(ws.codes_b().cpu().numpy(), want_b)
+    assert ws.scalar("step_a").item() == float(sa) and ws.scalar("step_b").item() == float(sb)
+    rng = np.random.default_rng(0)
+    rows = np.sort(rng.choice(M, 64, replace=False))
+    cols = np.sort(rng.choice(N, 64, replace=False))
+    got = out.cpu().numpy()
+    want_rows, _, _ = O.gemm_i8_tiled(want_a[rows], want_b, sa, sb)
+    want_cols, _, _ = O.gemm_i8_tiled(want_a, want_b[cols], sa, sb)
+    _assert_close(got[rows], want_rows)
+    _assert_close(got[:, cols], want_cols)
+    assert np.array_equal(got[rows], want_rows) and np.array_equal(got[:, cols], want_cols)

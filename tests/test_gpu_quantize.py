@@ -1,0 +1,138 @@
+"""GPU parity: FWHT + calibration maximum + quantizer against the CPU oracle (bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hdqt_oracle as O
+from paper_2310_03675_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def hdqt():
+    from paper_2310_03675_b200 import hdqt as mod
+    return mod
+
+
+def _dev(x):
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def _expected_norms(codes):
+    rows, Kp = codes.shape
+    sq = (codes.astype(np.int64) ** 2).reshape(rows, Kp // 32, 32).sum(2)
+    nb = (rows + 127) // 128
+    out = np.zeros((nb, Kp // 32), dtype=np.int64)
+    for b in range(nb):
+        out[b] = sq[b * 128:(b + 1) * 128].max(0)
+    return out
+
+
+SHAPES = [(32, 128), (32, 64), (1, 32), (7, 27), (129, 100), (300, 561), (256, 1152), (1000, 96), (5, 8)]
+
+
+@pytest.mark.parametrize("rows,K", SHAPES)
+@pytest.mark.parametrize("layout", ["k_contiguous", "k_strided"])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantize_matches_oracle(hdqt, rows, K, layout, mode):
+    x = inputs.gradients(rows, K, seed=rows * 1000 + K, scale=1.0)
+    want_codes, want_step, want_amax = O.quantize_hadamard(x, 32, 4, 1.0, mode, seed=5, tag=9)
+    if layout == "k_contiguous":
+        src = _dev(x)
+    else:
+        src = _dev(x.T).t()            # same logical [rows, K], rows contiguous in memory
+    status = hdqt.new_status("cuda")
+    amax = hdqt.absmax_hadamard(src, 32, status)
+    codes, step, norms = hdqt.quantize_hadamard(src, 32, 4, 1.0, mode, seed=5, tag=9, want_norms=True,
+                                                dev_status=status)
+    hdqt.check_device_status(status)
+    assert amax.item() == float(want_amax)
+    assert step.item() == float(want_step)
+    got = codes.cpu().numpy()
+    assert got.shape == want_codes.shape
+    assert np.array_equal(got, want_codes)
+    assert np.array_equal(norms.cpu().numpy().astype(np.int64), _expected_norms(want_codes))
+
+
+@pytest.mark.parametrize("bits,clip,had", [(2, 1.0, 32), (3, 0.975, 32), (5, 1.0, 16), (6, 0.5, 8), (8, 0.975, 32),
+                                           (8, 0.25, 4), (4, 0.975, 1), (4, 1.0, 2)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_bit_widths_clip_and_block_sizes(hdqt, bits, clip, had, mode):
+    x = inputs.activations(70, 200, seed=bits * 10 + had)
+    want_codes, want_step, _ = O.quantize_hadamard(x, had, bits, clip, mode, seed=77, tag=3)
+    for src in (_dev(x), _dev(x.T).t()):
+        codes, step, _ = hdqt.quantize_hadamard(src, had, bits, clip, mode, seed=77, tag=3)
+        assert step.item() == float(want_step)
+        assert np.array_equal(codes.cpu().numpy(), want_codes)
+
+
+def test_unaligned_row_stride_and_views(hdqt):
+    base = inputs.activations(64, 203, seed=1)
+    x = base[:, 3:130]                       # K = 127, row stride 203 (not a multiple of 4), offset pointer
+    want, step_w, _ = O.quantize_hadamard(x, 32, 4, 1.0, 1, seed=1, tag=1)
+    src = _dev(base)[:, 3:130]
+    codes, step, _ = hdqt.quantize_hadamard(src, 32, 4, 1.0, 1, seed=1, tag=1)
+    assert step.item() == float(step_w)
+    assert np.array_equal(codes.cpu().numpy(), want)
+
+
+def test_supplied_amax_skips_calibration(hdqt):
+    x = inputs.activations(40, 96, seed=2)
+    amax = np.float32(123.5)
+    xh = O.fwht_blockdiag(O.pad_contraction(x, 32), 32)
+    want, want_step, _ = O.quantize_transformed(xh, 4, 0.975, 0, amax=amax)
+    codes, step, _ = hdqt.quantize_hadamard(_dev(x), 32, 4, 0.975, 0, amax=torch.tensor([amax], device="cuda"))
+    assert step.item() == float(want_step)
+    assert np.array_equal(codes.cpu().numpy(), want)
+
+
+def test_seed_high_word_and_determinism(hdqt):
+    x = _dev(inputs.gradients(64, 64, seed=3))
+    a, _, _ = hdqt.quantize_hadamard(x, mode=1, seed=(5 << 32) + 1, tag=2)
+    b, _, _ = hdqt.quantize_hadamard(x, mode=1, seed=(5 << 32) + 1, tag=2)
+    c, _, _ = hdqt.quantize_hadamard(x, mode=1, seed=1, tag=2)
+    assert torch.equal(a, b) and not torch.equal(a, c)
+    want, _, _ = O.quantize_hadamard(x.cpu().numpy(), 32, 4, 1.0, 1, seed=(5 << 32) + 1, tag=2)
+    assert np.array_equal(a.cpu().numpy(), want)
+
+
+def test_all_zero_and_nonfinite(hdqt):
+    status = hdqt.new_status("cuda")
+    z = torch.zeros(16, 64, device="cuda")
+    codes, step, _ = hdqt.quantize_hadamard(z, dev_status=status)
+    assert not codes.any().item() and step.item() == 0.0 and status.item() == 0
+    z[3, 5] = float("inf")
+    hdqt.quantize_hadamard(z, dev_status=status)
+    assert status.item() == 5          # HDQT_ERR_NONFINITE, reported through the device status word
+    status.zero_()
+    z[3, 5] = float("nan")
+    hdqt.absmax_hadamard(z.t().contiguous().t(), dev_status=status)
+    assert status.item() == 5
+
+
+def test_output_canaries(hdqt):
+    """Nothing is written outside [rows, K_pad]."""
+    rows, K = 37, 70
+    Kp = hdqt.padded_k(K)
+    buf = torch.full((rows * Kp + 512,), 0x5A, dtype=torch.int8, device="cuda")
+    codes = buf[256:256 + rows * Kp].view(rows, Kp)
+    step = torch.empty(1, device="cuda")
+    ws = torch.empty(hdqt.lib.hdqt_quantize_workspace_bytes(rows, K, 32), dtype=torch.uint8, device="cuda")
+    x = _dev(inputs.activations(rows, K, seed=4))
+    for src in (x, x.t().contiguous().t()):
+        hdqt.quantize_hadamard(src, mode=1, out=(codes, step, None, ws))
+        torch.cuda.synchronize()
+        assert (buf[:256] == 0x5A).all().item() and (buf[256 + rows * Kp:] == 0x5A).all().item()
+
+
+def test_large_tensor_multiple_waves(hdqt):
+    """Larger than one grid wave, ragged tail; codes compared in full."""
+    rows, K = 3001, 2080
+    x = inputs.heavy_tailed(rows, K, seed=8)
+    for mode in (0, 1):
+        want, step_w, _ = O.quantize_hadamard(x, 32, 4, 1.0, mode, seed=2, tag=4)
+        for src in (_dev(x), _dev(x.T).t()):
+            codes, step, _ = hdqt.quantize_hadamard(src, mode=mode, seed=2, tag=4)
+            assert step.item() == float(step_w)
+            assert np.array_equal(codes.cpu().numpy(), want)
