@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the HDQT quantized training GEMM hot path on B200.
+
+One "step" = one pass of the whole path over one synthetic batch:
+  calibration maximum + FWHT + quantize of both operands -> tiled int8 tensor-core GEMM with
+  8-bit per-tile accumulators -> wide tile sum -> dequantising epilogue.
+Workload = one shape of the roofline sweep (dgrad layout: A K-contiguous with stochastic
+rounding, B K-contiguous with nearest rounding), operands Student-t(3) with 0.1 % outliers x50.
+
+Prints ONE JSON line (see README for the keys).  `--impl reference` times the CPU
+oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "hdqt_gemm_int_tops"
+UNIT = "TOPS"
+SEED = 1234
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="hdqt", choices=["hdqt", "reference"])
+    ap.add_argument("--size", type=int, default=8192, help="M = N = K of the sweep shape")
+    ap.add_argument("--no-merge", action="store_true", help="disable merging of provably clamp-free tiles")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def workload_config(size: int, merge: bool):
+    return {
+        "workload": f"roofline-sweep dgrad-layout HDQT GEMM M=N=K={size} (Student-t(3), 0.1% outliers x50)",
+        "M": size, "N": size, "K": size,
+        "in_bits": 4, "acc_bits": 8, "acc_tile": 32, "had_block": 32, "acc_shift": 0,
+        "rounding": "A stochastic (Philox4x32-10), B nearest",
+        "clamp_free_tile_merging": bool(merge),
+        "l2": "inputs_exceed_l2" if size * size * 4 > 126 * 2 ** 20 else "inputs_within_l2_not_flushed",
+        "parallelism": "replicas",
+    }
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample_run(size: int, rows_a: int, rows_b: int, seed: int):
+    """One pass of the oracle over a slice of the workload: rows_a rows of A, rows_b rows of B, full K.
+    Returns (seconds, equivalent integer ops)."""
+    from oracle import hdqt_oracle as O
+    from paper_2310_03675_b200 import inputs
+    A = inputs.heavy_tailed(rows_a, size, seed)
+    B = inputs.heavy_tailed(rows_b, size, seed + 1)
+    t0 = time.perf_counter()
+    O.gemm_dgrad(A, B, O.dgrad_desc(seed=seed))
+    dt = time.perf_counter() - t0
+    return dt, 2.0 * rows_a * rows_b * size
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(size: int):
+    rows_a, rows_b = min(size, 1024), min(size, 2048)
+    dt, ops = oracle_sample_run(size, rows_a, rows_b, SEED)
+    return {"value": ops / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "seconds": dt,
+            "sample": f"{rows_a} rows of A x {rows_b} rows of B, full K={size} (whole path: FWHT, quantize, "
+                      f"tiled GEMM, dequant); ops counted as 2*rows_a*rows_b*K"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    size = args.size
+    rows_a, rows_b = min(size, 256), min(size, 512)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_run(size, rows_a, rows_b, SEED)
+    total_t, total_ops = 0.0, 0.0
+    for i in range(args.steps):
+        dt, ops = oracle_sample_run(size, rows_a, rows_b, SEED + i)
+        total_t += dt
+        total_ops += ops
+    value = total_ops / total_t / 1e12
+    sample = f"each step: {rows_a} rows of A x {rows_b} rows of B, full K={size}, whole path on the CPU oracle"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_t / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32", "data": "synthetic",
+        "config": workload_config(size, not args.no_merge),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+
+def run_hdqt(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2310_03675_b200 import hdqt, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    size = args.size
+    M = N = K = size
+    merge = not args.no_merge
+    flags = 0 if merge else hdqt.FLAG_NO_MERGE
+    desc = hdqt.default_desc("dgrad", seed=SEED, flags=flags)
+
+    # every rank works on its own operands (independent problems: no data-path collective)
+    A = inputs.heavy_tailed_torch(M, K, SEED + 10 * rank, dev)
+    B = inputs.heavy_tailed_torch(N, K, SEED + 10 * rank + 1, dev)
+    out = torch.empty((M, N), dtype=torch.float32, device=dev)
+    status = hdqt.new_status(dev)
+    Kp = hdqt.padded_k(K)
+
+    # stage-level buffers (the same launches the composite call makes, with events between stages)
+    def qbufs(rows):
+        return (torch.empty((rows, Kp), dtype=torch.int8, device=dev), torch.empty(1, device=dev),
+                torch.empty(((rows + 127) // 128, Kp // 32), dtype=torch.int32, device=dev) if merge else None,
+                torch.empty(hdqt.lib.hdqt_quantize_workspace_bytes(rows, K, 32), dtype=torch.uint8, device=dev))
+    bufA, bufB = qbufs(M), qbufs(N)
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        hdqt.quantize_hadamard(A, 32, desc.in_bits, desc.clip_a, desc.round_a, desc.seed, desc.tag_a,
+                               want_norms=merge, dev_status=status, out=bufA)
+        hdqt.quantize_hadamard(B, 32, desc.in_bits, desc.clip_b, desc.round_b, desc.seed, desc.tag_b,
+                               want_norms=merge, dev_status=status, out=bufB)
+        if ev:
+            ev[1].record(stream)
+        hdqt.gemm_i8_tiled(bufA[0], bufB[0], bufA[1], bufB[1], desc.acc_bits, desc.acc_tile, desc.acc_shift,
+                           desc.had_block, norms_a=bufA[2], norms_b=bufB[2], flags=flags, dev_status=status, out=out)
+        if ev:
+            ev[2].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    hdqt.check_device_status(status, "warm-up")
+
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(events[i])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    hdqt.check_device_status(status, "timed region")
+    elapsed_ms = t_start.elapsed_time(t_end)
+    quant_ms = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
+    gemm_ms = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
+
+    # end to end through the public call with host buffers: H2D of both operands, D2H of the result
+    e2e = None
+    if not args.skip_e2e:
+        hA = torch.empty((M, K), dtype=torch.float32).pin_memory()
+        hB = torch.empty((N, K), dtype=torch.float32).pin_memory()
+        hA.copy_(A)
+        hB.copy_(B)
+        hOut = torch.empty((M, N), dtype=torch.float32).pin_memory()
+        dA, dB = torch.empty_like(A), torch.empty_like(B)
+        ws = hdqt.Workspace(desc, M, N, K, dev)
+        e2e_steps = max(3, min(args.steps, 5))
+
+        def e2e_step():
+            dA.copy_(hA, non_blocking=True)
+            dB.copy_(hB, non_blocking=True)
+            hdqt.gemm_dgrad(dA, dB, desc=desc, workspace=ws, dev_status=status, out=out)
+            hOut.copy_(out, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = t.item()
+        e2e = {"value": world * e2e_steps * 2.0 * M * N * K / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": hA.numel() * 4 + hB.numel() * 4, "d2h_bytes_per_step": hOut.numel() * 4,
+               "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps}
+        hdqt.check_device_status(status, "e2e")
+
+    if world > 1:
+        t = torch.tensor([elapsed_ms, quant_ms, gemm_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, quant_ms, gemm_ms = t.tolist()
+
+    if rank == 0:
+        peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(peaks_path):
+            peaks = json.load(open(peaks_path))
+            bf16_sustained = peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops"))
+            hbm = peaks["hbm_gbs"]
+            peak_src = "measured bf16 sustained x2 (nominal int8:bf16 ratio)"
+        else:
+            bf16_sustained, hbm = 1400.0, 6650.0
+            peak_src = "fallback bf16 sustained x2 (nominal int8:bf16 ratio)"
+        int8_peak = 2.0 * bf16_sustained
+        ops = 2.0 * M * N * K
+        gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
+        quant_bytes = 9.0 * (M * K + N * K)      # 4 B calibration read + 4 B read + 1 B code written, per element
+        line = {
+            "metric": METRIC, "value": world * args.steps * ops / (elapsed_ms * 1e-3) / 1e12, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32",
+            "data": "synthetic", "config": workload_config(size, merge),
+            "roofline": {"bound": "tensor", "kernel": "gemm_i8_tiled_kernel", "achieved": gemm_tops,
+                         "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak, "peak_source": peak_src,
+                         "traffic": None, "ms_per_launch": gemm_ms},
+            "quantize": {"ms_per_step": quant_ms, "algorithmic_gb_per_step": quant_bytes / 1e9,
+                         "gbs": quant_bytes / (quant_ms * 1e-3) / 1e9, "hbm_peak_gbs": hbm,
+                         "frac": quant_bytes / (quant_ms * 1e-3) / 1e9 / hbm,
+                         "note": "both operands: calibration pass (4 B/elt) + FWHT/quantize pass (5 B/elt)"},
+            "clocks": clocks, "gpu_launches": args.steps * (5 + (2 if merge else 0)),
+        }
+        if e2e is not None:
+            line["e2e"] = e2e
+        if not args.skip_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(size)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_hdqt(args)
+
+
+if __name__ == "__main__":
+    main()

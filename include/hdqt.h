@@ -159,8 +159,10 @@ size_t hdqt_quantize_workspace_bytes(int64_t rows, int64_t K, int32_t had_block)
  *   S = sum over tiles t of clamp(rne(P_t / 2^r), -2^(b_a-1), 2^(b_a-1)-1),
  *   P_t[m, n] = sum over the tile's k of Aq[m, k]*Bq[n, k]          (exact).
  *
- * Aq [M, K_pad], Bq [N, K_pad]: int8 codes, K contiguous, K_pad % 32 == 0,
- *     |code| <= 2^(bits-1) with bits <= 8.
+ * Aq [M, K_pad], Bq [N, K_pad]: int8 codes, K contiguous, K_pad % 32 == 0.
+ * code_bits: the caller's promise that every |code| <= 2^(code_bits-1) (2..8; 8 is always
+ *     true).  It bounds the tile sums and selects the narrowest exact epilogue; codes that
+ *     break the promise give undefined results.
  * step_a, step_b: device scalars written by hdqt_quantize_hadamard.
  * out   : fp32 [M, ld_out] row-major, ld_out >= N.
  * S_out : optional int32 [M, N] (dense): the integer sums S.
@@ -177,7 +179,7 @@ size_t hdqt_quantize_workspace_bytes(int64_t rows, int64_t K, int32_t had_block)
  */
 hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, const float* step_a,
                                  const float* step_b, int64_t M, int64_t N, int64_t K_pad,
-                                 int32_t acc_bits, int32_t acc_tile, int32_t acc_shift,
+                                 int32_t code_bits, int32_t acc_bits, int32_t acc_tile, int32_t acc_shift,
                                  int32_t had_block, float* out, int64_t ld_out,
                                  int32_t* S_out, void* tiles_out, int32_t tiles_elem_bytes,
                                  const int32_t* norms_a, const int32_t* norms_b,

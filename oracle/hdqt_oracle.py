@@ -148,6 +148,23 @@ def sr_random_u16(seed: int, tag: int, idx: np.ndarray) -> np.ndarray:
     return half.astype(np.int64)
 
 
+def sr_random_u16_tensor(seed: int, tag: int, rows: int, K_pad: int) -> np.ndarray:
+    """sr_random_u16 for every element of a [rows, K_pad] code tensor, with one
+    Philox call per group of eight elements instead of one per element."""
+    n = rows * K_pad
+    assert n % 8 == 0
+    g = np.arange(n // 8, dtype=np.uint64)
+    w = philox4x32_10(g & _MASK32, g >> np.uint64(32),
+                      np.full(g.shape, int(tag) & 0xFFFFFFFF, dtype=np.uint64),
+                      np.zeros(g.shape, dtype=np.uint64),
+                      int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF)
+    out = np.empty((n // 8, 8), dtype=np.int64)
+    for j in range(4):
+        out[:, 2 * j] = w[j] & np.uint32(0xFFFF)       # even element: low half of word j
+        out[:, 2 * j + 1] = w[j] >> np.uint32(16)      # odd element: high half
+    return out.reshape(rows, K_pad)
+
+
 # --------------------------------------------------------------------------
 # Quantizer (Section 3, definition of Q; Section 4, clip factor 0.975)
 # --------------------------------------------------------------------------
@@ -191,9 +208,7 @@ def quantize_transformed(xh: np.ndarray, bits: int, clip: float, mode: int,
     elif mode == ROUND_STOCHASTIC:
         v_fx = np.rint((v * F32(65536.0)).astype(F32)).astype(np.int64)
         rows, Kp = xh.shape
-        idx = (np.arange(rows, dtype=np.uint64)[:, None] * np.uint64(Kp)
-               + np.arange(Kp, dtype=np.uint64)[None, :])
-        u16 = sr_random_u16(seed, tag, idx)
+        u16 = sr_random_u16_tensor(seed, tag, rows, Kp)
         q = (v_fx + u16) >> 16          # arithmetic shift = floor division
     else:
         raise ValueError("unknown rounding mode")

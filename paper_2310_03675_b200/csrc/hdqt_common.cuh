@@ -3,6 +3,8 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "hdqt.h"
 
@@ -57,6 +59,12 @@ __device__ __forceinline__ QuantScale make_quant_scale(float amax, float clip, i
   q.bad = !(isfinite(amax)) || (!q.zero && !isfinite(q.m));
   if (q.zero || q.bad) { q.m = 0.0f; q.step = 0.0f; }
   return q;
+}
+
+// A failed CUDA call: HDQT_ERR_CUDA, with the runtime's message on stderr when HDQT_DEBUG is set.
+inline hdqt_status_t cuda_failure(cudaError_t e, const char* what) {
+  if (getenv("HDQT_DEBUG") != nullptr) fprintf(stderr, "[hdqt] %s: %s\n", what, cudaGetErrorString(e));
+  return HDQT_ERR_CUDA;
 }
 
 // ---- internal launchers (defined in the .cu files) ----

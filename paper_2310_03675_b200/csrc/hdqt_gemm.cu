@@ -8,11 +8,14 @@
 //   out      = fp32(S) * fp32(step_a*step_b*2^r / n_h)
 //
 // One CTA owns a 128 x 256 output block.  Warp 0 feeds a 4-stage shared-memory ring with TMA
-// (128-byte swizzled rows = 4 tiles of 32 k per stage), warp 1 issues the MMAs into a TMEM
-// accumulator ring of 2 x 256 columns, warps 2..9 drain the accumulators (tcgen05.ld), apply
-// the accumulator quantisation per tile and keep the wide sums in registers.
+// (128-byte swizzled rows = 4 tiles of 32 k per stage), warp 1 issues the MMAs into two TMEM
+// accumulators of 256 columns, warps 2..17 drain the accumulators (tcgen05.ld), apply the
+// accumulator quantisation per tile and keep the wide sums in registers.
+// Tiles that provably cannot clamp (Cauchy-Schwarz bound from per-tile code norms) may be
+// accumulated together in TMEM: the clamp is the identity there, so the integers are unchanged.
 // Every wait is bounded; when one runs out the CTA records HDQT_ERR_TIMEOUT and leaves.
 #include <cuda.h>
+#include <string.h>
 
 #include "hdqt_common.cuh"
 
@@ -27,10 +30,12 @@ constexpr int STAGES = 4;
 constexpr int A_STAGE = BM * BKB;              // 16 KB
 constexpr int B_STAGE = BN * BKB;              // 32 KB
 constexpr int STAGE_BYTES = A_STAGE + B_STAGE; // 48 KB
-constexpr int NUM_EPI_WARPS = 8;
+constexpr int NUM_EPI_WARPS = 16;              // 4 per TMEM lane quarter, 64 accumulator columns each
+constexpr int EPI_COLS = BN / (NUM_EPI_WARPS / 4);
 constexpr int GEMM_THREADS = 32 * (2 + NUM_EPI_WARPS);
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int MAX_CERT_WORDS = 512;            // certificate bitmask: up to 16384 accumulator tiles
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 4 * MAX_CERT_WORDS;
 
 // instruction descriptor: D = s32, A = B = signed 8-bit, both K-major, N = 256, M = 128
 constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
@@ -40,9 +45,17 @@ struct GemmParams {
   int64_t M, N, K_pad;
   int32_t tiles32;        // K_pad / 32
   int32_t tiles_per_acc;  // acc_tile / 32 (tiles32 if acc_tile == 0)
+  int32_t num_acc;        // accumulator tiles along K
   int32_t acc_shift;
   int32_t lo, hi;         // accumulator range
   int32_t had_block;
+  int32_t flush_every;    // packed mode: accumulator tiles summed in 16-bit lanes before widening
+  // merging of provably clamp-free accumulator tiles
+  int32_t merge;          // 0 = off, 1 = certificates from the tile norms, 2 = every tile is clamp-free
+  int32_t merge_max_uncert_256;  // a CTA merges only if uncertified tiles <= this/256 of all tiles
+  int64_t cert_thr_sq;    // a 32-wide sub-tile is certified iff norm_a*norm_b <= this
+  const int32_t* norms_a; // [ceil(M/128), tiles32]
+  const int32_t* norms_b; // [ceil(N/128), tiles32]
   const float* step_a;
   const float* step_b;
   float* out;
@@ -51,6 +64,8 @@ struct GemmParams {
   void* tiles_out;
   int32_t tiles_elem_bytes;
   int32_t* dev_status;
+  int32_t debug_mode;
+  long long* debug_ts;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -80,15 +95,47 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after ~1 s, or as soon as another role has given up.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded waits: each gives up after ~1 s, or as soon as another role has given up.
+//
+// mbar_wait: for the two single-thread roles (TMA producer, MMA issuer), whose waits are on the
+// critical path of every K tile: polls without suspending first, then backs off.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (int i = 0; i < (1 << 14); ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+  for (int i = 0; i < (1 << 12); ++i) {
+    if (mbar_test_wait(bar, parity)) return true;
   }
   for (int i = 0; i < (1 << 20); ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     __nanosleep(512);
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// mbar_wait_yield: for the epilogue warps. A warp that spins steals issue slots from the MMA issuer
+// and from the warps that have work, so these waits suspend in hardware (try_wait) and sleep between
+// polls; kSleepNs is the poll period (short for the per-tile handshake, long for the one wait on the
+// merged accumulator that spans the whole main loop).
+template <int kSleepNs>
+__device__ __forceinline__ bool mbar_wait_yield(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  constexpr int kLimit = (kSleepNs >= 512) ? (1 << 21) : (1 << 24);
+  for (int i = 0; i < kLimit; ++i) {
+    __nanosleep(kSleepNs);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63) == 63 && *abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
@@ -145,6 +192,49 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
 
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+#define HDQT_TMEM_LD32_PACK16(taddr, v)                                                                 \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x32.pack::16b.b32 "                                               \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                         \
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"         \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),      \
+        "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),      \
+        "=r"(v[29]), "=r"(v[30]), "=r"(v[31])                                                           \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
+#define HDQT_TMEM_LD16_PACK16(taddr, v)                                                                 \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x16.pack::16b.b32 "                                               \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"                  \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15])                                                                                     \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
+// tcgen05.wait::ld tied to the registers of the load it completes, so that the compiler cannot move
+// their first use above the wait
+#define HDQT_TMEM_WAIT16(v)                                                                             \
+  asm volatile("tcgen05.wait::ld.sync.aligned;"                                                         \
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]),    \
+                 "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), \
+                 "+r"(v[14]), "+r"(v[15])                                                               \
+               :                                                                                        \
+               : "memory")
+
+#define HDQT_TMEM_LD16(taddr, v)                                                                        \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "                                                         \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"                  \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15])                                                                                     \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
 // accumulator quantisation of one exact tile sum
 template <bool kShift>
 __device__ __forceinline__ int acc_quant(int P, int r, int lo, int hi) {
@@ -155,9 +245,52 @@ __device__ __forceinline__ int acc_quant(int P, int r, int lo, int hi) {
   return min(max(P, lo), hi);
 }
 
-// ---- the kernel -----------------------------------------------------------------------------
+// Writes 4 consecutive output columns of one row: the final fp32 values (and optionally the integer
+// sums), or - for an intermediate widening of the packed sums - the int32 partial sums, which are
+// parked in the output buffer itself until the final pass reads them back.
+template <bool kFinal>
+__device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t gn, int (&s)[4], bool have_prev,
+                                      bool vec, float scale) {
+  float* orow = p.out + gm * p.ld_out + gn;
+  if (vec) {
+    if (have_prev) {
+      const int4 prev = *reinterpret_cast<const int4*>(orow);
+      s[0] += prev.x; s[1] += prev.y; s[2] += prev.z; s[3] += prev.w;
+    }
+    if (kFinal) {
+      float4 o;
+      o.x = __fmul_rn((float)s[0], scale);
+      o.y = __fmul_rn((float)s[1], scale);
+      o.z = __fmul_rn((float)s[2], scale);
+      o.w = __fmul_rn((float)s[3], scale);
+      *reinterpret_cast<float4*>(orow) = o;
+    } else {
+      *reinterpret_cast<int4*>(orow) = make_int4(s[0], s[1], s[2], s[3]);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (gn + i < p.N) {
+        if (have_prev) s[i] += __float_as_int(orow[i]);
+        orow[i] = kFinal ? __fmul_rn((float)s[i], scale) : __int_as_float(s[i]);
+      }
+    }
+  }
+  if (kFinal && p.S_out != nullptr) {
+    int32_t* srow = p.S_out + gm * p.N + gn;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (gn + i < p.N) srow[i] = s[i];
+    }
+  }
+}
 
-template <bool kShift, bool kTilesOut>
+// ---- the kernel -----------------------------------------------------------------------------
+// kPacked: the per-tile sums fit 16 bits and b_a <= 8, r = 0: TMEM is read with two columns packed
+//          per register, clamp and add work on 16-bit lane pairs (half the ALU work per element).
+// otherwise: one 32-bit register per accumulator element, any b_a and r.
+
+template <bool kPacked, bool kShift, bool kTilesOut>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const GemmParams p) {
@@ -172,13 +305,15 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   const uint32_t bar_tempty = bar_tfull + 16;           // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* s_uncert = reinterpret_cast<int*>(tmem_slot + 2);
+  uint32_t* cert_mask = reinterpret_cast<uint32_t*>(smem_al + STAGES * STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * BM;
   const int n0 = blockIdx.y * BN;
   const int num_kblocks = (p.tiles32 + 3) >> 2;
-  const int num_acc = (p.tiles32 + p.tiles_per_acc - 1) / p.tiles_per_acc;
+  const int num_acc = p.num_acc;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -190,6 +325,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       mbar_init(bar_tempty + 8 * b, NUM_EPI_WARPS);
     }
     *abort_flag = 0;
+    *s_uncert = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -204,6 +340,49 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // ---- which accumulator tiles provably cannot clamp (Cauchy-Schwarz on the tile norms) ----
+  // bit a of cert_mask is set iff every 32-wide sub-tile of accumulator tile a satisfies
+  // max_row ||a||^2 * max_col ||b||^2 <= (hi / tiles_per_acc)^2, so |P| <= hi for the whole block.
+  if (p.merge == 1) {
+    if (warp >= 2) {
+      const int et = threadIdx.x - 64;
+      const int64_t T = p.tiles32;
+      const int32_t* na = p.norms_a + (int64_t)blockIdx.x * T;
+      const int64_t nb_blk = (int64_t)blockIdx.y * 2;
+      const int32_t* nb0 = p.norms_b + nb_blk * T;
+      const bool has1 = (nb_blk + 1) * 128 < p.N;
+      const int32_t* nb1 = nb0 + T;
+      int my_uncert = 0;
+      const int acc_round = (num_acc + 31) & ~31;
+      for (int a = et; a < acc_round; a += 32 * NUM_EPI_WARPS) {
+        bool cert = false;
+        if (a < num_acc) {
+          cert = true;
+          const int t0 = a * p.tiles_per_acc;
+          const int t1 = min(p.tiles32, t0 + p.tiles_per_acc);
+          for (int t = t0; t < t1; ++t) {
+            const int64_t a2 = __ldg(na + t);
+            int64_t b2 = __ldg(nb0 + t);
+            if (has1) b2 = max(b2, (int64_t)__ldg(nb1 + t));
+            cert = cert && (a2 * b2 <= p.cert_thr_sq);
+          }
+          my_uncert += cert ? 0 : 1;
+        }
+        const uint32_t bits = __ballot_sync(0xFFFFFFFFu, cert);
+        if (lane == 0) cert_mask[a >> 5] = bits;
+      }
+      my_uncert = __reduce_add_sync(0xFFFFFFFFu, my_uncert);
+      if (lane == 0 && my_uncert) atomicAdd(s_uncert, my_uncert);
+    }
+    __syncthreads();
+  }
+  const int n_uncert = (p.merge == 2) ? 0 : *s_uncert;
+  // merge in this CTA only when few tiles need the clamp path (it is single-buffered when merging)
+  const bool merging = (p.merge == 2) ||
+                       (p.merge == 1 && (int64_t)n_uncert * 256 <= (int64_t)p.merge_max_uncert_256 * num_acc);
+  const int n_clamp_tiles = merging ? n_uncert : num_acc;
+  const int n_merged = merging ? num_acc - n_uncert : 0;
+
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
@@ -212,6 +391,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const int s = kb % STAGES;
         const uint32_t par = ((kb / STAGES) & 1) ^ 1;
         if (!mbar_wait(bar_empty + 8 * s, par, abort_flag)) break;
+        if (p.debug_mode & 2) { mbar_arrive(bar_full + 8 * s); issued = kb + 1; continue; }
         mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
         const uint32_t a_dst = smem_base + s * STAGE_BYTES;
         tma_load_2d(a_dst, &map_a, kb * BKB, m0, bar_full + 8 * s);
@@ -230,95 +410,260 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
     if (lane == 0) {
-      for (int kt = 0; kt < p.tiles32; ++kt) {
-        const int kb = kt >> 2, sub = kt & 3;
-        const int s = kb % STAGES;
-        if (sub == 0) {
-          if (!mbar_wait(bar_full + 8 * s, (kb / STAGES) & 1, abort_flag)) break;
-        }
-        const int acc = kt / p.tiles_per_acc;
-        const int j = kt - acc * p.tiles_per_acc;
-        const int buf = acc & 1;
-        if (j == 0) {
-          if (!mbar_wait(bar_tempty + 8 * buf, ((acc >> 1) & 1) ^ 1, abort_flag)) break;
-        }
+      // tcgen05.mma holds the issuing thread until the tensor pipe takes the operation, and the pipe
+      // idles while this thread does anything else: bookkeeping between two MMAs is dead tensor time.
+      // Stages whose four tiles are all merged are therefore issued as four back-to-back MMAs, with
+      // the next stage's barrier polled ahead; only stages with clamp tiles take the per-tile code.
+      const uint64_t desc_a0 = make_smem_desc(smem_base);
+      const uint64_t desc_b0 = make_smem_desc(smem_base + A_STAGE);
+      int s = 0;                 // smem stage
+      uint32_t full_par = 0;     // parity of the stage's next "full" phase
+      int j = 0;                 // position inside the current accumulator tile
+      int acc = 0;               // accumulator tile index
+      int clamp_idx = 0;         // index among the tiles that take the clamp path
+      bool cert = (p.merge == 2);
+      uint32_t merged_started = 0;
+      uint32_t d_tmem = tmem_base;
+      uint32_t tfull_bar = bar_tfull;
+      uint64_t desc_a = desc_a0, desc_b = desc_b0;
+      bool ok = true;
+      const int tiles32 = p.tiles32, tpa = p.tiles_per_acc;
+      const bool nibble_ok = (p.merge == 2) || (merging && tpa == 1);
+      bool ready = mbar_test_wait(bar_full, 0u);
+      for (int kb = 0; kb < num_kblocks; ++kb) {
+        if (!ready && !mbar_wait(bar_full + 8 * s, full_par, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t a_addr = smem_base + s * STAGE_BYTES + sub * 32;
-        const uint64_t a_desc = make_smem_desc(a_addr);
-        const uint64_t b_desc = make_smem_desc(a_addr + A_STAGE);
-        tc_mma_i8(tmem_base + buf * BN, a_desc, b_desc, j != 0);
-        const bool last = (kt == p.tiles32 - 1);
-        if (j == p.tiles_per_acc - 1 || last) tc_commit(bar_tfull + 8 * buf);
-        if (sub == 3 || last) tc_commit(bar_empty + 8 * s);
+        // poll the next stage now; the answer is needed only after this stage's MMAs
+        const int s_next = (s + 1 == STAGES) ? 0 : s + 1;
+        const uint32_t par_next = (s + 1 == STAGES) ? (full_par ^ 1u) : full_par;
+        const int kt0 = kb * 4;
+        uint32_t nib = 0;
+        if (p.merge == 2) nib = 0xFu;
+        else if (nibble_ok) nib = (cert_mask[kb >> 3] >> ((kb & 7) * 4)) & 0xFu;
+        if (nib == 0xFu && kt0 + 4 <= tiles32) {
+          tc_mma_i8(tmem_base, desc_a, desc_b, merged_started);
+          tc_mma_i8(tmem_base, desc_a + 2, desc_b + 2, 1u);
+          tc_mma_i8(tmem_base, desc_a + 4, desc_b + 4, 1u);
+          tc_mma_i8(tmem_base, desc_a + 6, desc_b + 6, 1u);
+          merged_started = 1u;
+          acc += 4;    // only meaningful (and only used) when tiles_per_acc == 1
+        } else {
+          const int kt1 = min(tiles32, kt0 + 4);
+          for (int kt = kt0; kt < kt1; ++kt) {
+            if (j == 0) {
+              if (p.merge == 2) {
+                cert = true;
+              } else if (merging) {
+                cert = (cert_mask[acc >> 5] >> (acc & 31)) & 1u;
+              }
+              if (cert) {
+                d_tmem = tmem_base;                      // merged tiles accumulate in buffer 0
+              } else {
+                // clamp tiles: buffer 1 when merging, else alternate 0 / 1
+                const int buf = merging ? 1 : (clamp_idx & 1);
+                const uint32_t use = merging ? (uint32_t)clamp_idx : (uint32_t)(clamp_idx >> 1);
+                if (!mbar_wait(bar_tempty + 8 * buf, (use & 1) ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                d_tmem = tmem_base + buf * BN;
+                tfull_bar = bar_tfull + 8 * buf;
+              }
+            }
+            const uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
+            tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, cert ? merged_started : (uint32_t)(j != 0));
+            if (cert) merged_started = 1u;
+            if (++j == tpa || kt == tiles32 - 1) {
+              if (!cert) {
+                tc_commit(tfull_bar);
+                ++clamp_idx;
+              }
+              j = 0;
+              ++acc;
+            }
+          }
+          if (!ok) break;
+        }
+        tc_commit(bar_empty + 8 * s);
+        ready = (kb + 1 < num_kblocks) && mbar_test_wait(bar_full + 8 * s_next, par_next);
+        s = s_next;
+        full_par = par_next;
+        if (s == 0) {
+          desc_a = desc_a0;
+          desc_b = desc_b0;
+        } else {
+          desc_a += (uint64_t)(STAGE_BYTES >> 4);
+          desc_b += (uint64_t)(STAGE_BYTES >> 4);
+        }
       }
+      if (ok && n_merged > 0) tc_commit(bar_tfull + 0);
     }
   } else {
     // ------------------------------ epilogue warps ----------------------------
-    const int q = warp & 3;                 // TMEM lane quarter this warp may read
-    const int half = (warp - 2) >> 2;       // which 128 columns of the accumulator
+    const int q = warp & 3;                   // TMEM lane quarter this warp may read
+    const int grp = (warp - 2) >> 2;          // which EPI_COLS columns of the accumulator
     const int row = q * 32 + lane;
     const int64_t gm = (int64_t)m0 + row;
-    const int64_t gn0 = (int64_t)n0 + half * 128;
-    int S[128];
-#pragma unroll
-    for (int i = 0; i < 128; ++i) S[i] = 0;
+    const int64_t gn0 = (int64_t)n0 + grp * EPI_COLS;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(grp * EPI_COLS);
     const int r = p.acc_shift, lo = p.lo, hi = p.hi;
+    const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+                     (gn0 + EPI_COLS <= p.N);
     bool ok = true;
-    for (int acc = 0; acc < num_acc; ++acc) {
-      const int buf = acc & 1;
-      if (!mbar_wait(bar_tfull + 8 * buf, (acc >> 1) & 1, abort_flag)) { ok = false; break; }
-      tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * 128);
+
+    if (kPacked) {
+      // two columns per register: low half = even column, high half = odd column
+      uint32_t S[EPI_COLS / 2];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        HDQT_TMEM_LD32(taddr + c * 32, v);
-        tmem_ld_wait();
+      for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+      const uint32_t off = (uint32_t)(-lo);                    // c - lo lies in [0, hi - lo]
+      const uint32_t off2 = off | (off << 16);
+      const uint32_t rng2 = (uint32_t)(hi - lo) | ((uint32_t)(hi - lo) << 16);
+      int n_in_S = 0;
+      bool parked = false;   // int32 partial sums are parked in the output buffer
+      // Rolling pipeline over half-tiles (32 columns = 16 packed registers): while one half is clamped
+      // and added, the load of the next half (possibly of the next tile) is in flight.
+      uint32_t v0[EPI_COLS / 4], v1[EPI_COLS / 4];
+      if (n_clamp_tiles > 0) {
+        const int buf = merging ? 1 : 0;
+        if (!mbar_wait_yield<32>(bar_tfull + 8 * buf, 0u, abort_flag)) ok = false;
+        tc_fence_after();
+        if (ok) HDQT_TMEM_LD16_PACK16(lane_addr + buf * BN, v0);
+      }
+      for (int ci = 0; ci < n_clamp_tiles && ok; ++ci) {
+        const int buf = merging ? 1 : (ci & 1);
+        if (!(p.debug_mode & 8)) HDQT_TMEM_WAIT16(v0);                                         // first half of tile ci has landed
+        if (!(p.debug_mode & 8)) HDQT_TMEM_LD16_PACK16(lane_addr + buf * BN + EPI_COLS / 2, v1);  // second half in flight ...
+        if (!(p.debug_mode & 4)) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int ct = acc_quant<kShift>((int)v[i], r, lo, hi);
-          S[c * 32 + i] += ct;
-          if (kTilesOut) {
-            const int64_t n = gn0 + c * 32 + i;
-            if (gm < p.M && n < p.N) {
-              const int64_t off = ((int64_t)acc * p.M + gm) * p.N + n;
-              if (p.tiles_elem_bytes == 1) reinterpret_cast<int8_t*>(p.tiles_out)[off] = (int8_t)ct;
-              else reinterpret_cast<int16_t*>(p.tiles_out)[off] = (int16_t)ct;
+        for (int i = 0; i < EPI_COLS / 4; ++i) S[i] += __viaddmin_s16x2_relu(v0[i], off2, rng2);
+        }
+        if (!(p.debug_mode & 8)) HDQT_TMEM_WAIT16(v1);                                         // ... landed: the buffer is free
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+        if (p.debug_ts && blockIdx.x == 0 && blockIdx.y == 0 && warp == 2 && lane == 0 && ci >= 32 && ci < 96) p.debug_ts[(ci - 32) * 4 + 3] = clock64();
+        if (ci + 1 < n_clamp_tiles) {
+          const int nbuf = merging ? 1 : ((ci + 1) & 1);
+          const uint32_t use = merging ? (uint32_t)(ci + 1) : (uint32_t)((ci + 1) >> 1);
+          if (!mbar_wait_yield<32>(bar_tfull + 8 * nbuf, use & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          if (p.debug_ts && blockIdx.x == 0 && blockIdx.y == 0 && warp == 2 && lane == 0 && ci + 1 >= 32 && ci + 1 < 96) p.debug_ts[(ci + 1 - 32) * 4 + 2] = clock64();
+          if (!(p.debug_mode & 8)) HDQT_TMEM_LD16_PACK16(lane_addr + nbuf * BN, v0);           // first half of the next tile in flight
+        }
+        if (!(p.debug_mode & 4)) {
+#pragma unroll
+        for (int i = 0; i < EPI_COLS / 4; ++i) S[EPI_COLS / 4 + i] += __viaddmin_s16x2_relu(v1[i], off2, rng2);
+        }
+        if (++n_in_S == p.flush_every && ci + 1 < n_clamp_tiles) {
+          // widen: park int32 partial sums in the output buffer
+          if (gm < p.M) {
+#pragma unroll
+            for (int i = 0; i < EPI_COLS / 2; i += 2) {
+              int s4[4];
+              s4[0] = (int)(S[i] & 0xFFFFu) - (int)off * n_in_S;
+              s4[1] = (int)(S[i] >> 16) - (int)off * n_in_S;
+              s4[2] = (int)(S[i + 1] & 0xFFFFu) - (int)off * n_in_S;
+              s4[3] = (int)(S[i + 1] >> 16) - (int)off * n_in_S;
+              emit4<false>(p, gm, gn0 + 2 * i, s4, parked, vec, 0.0f);
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+          n_in_S = 0;
+          parked = true;
+        }
+      }
+      if (ok && n_merged > 0) {
+        ok = mbar_wait_yield<1000>(bar_tfull + 0, 0u, abort_flag);
+        tc_fence_after();
+      }
+      if (ok) {
+        const float scale = (float)((double)__ldg(p.step_a) * (double)__ldg(p.step_b) *
+                                    (double)(1u << p.acc_shift) / (double)p.had_block);
+#pragma unroll
+        for (int c = 0; c < EPI_COLS / 16; ++c) {
+          uint32_t mv[16];
+          if (n_merged > 0) {   // uniform
+            HDQT_TMEM_LD16(lane_addr + c * 16, mv);
+            HDQT_TMEM_WAIT16(mv);
+          }
+          if (gm < p.M) {
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) {
+              const uint32_t s0 = S[c * 8 + i], s1 = S[c * 8 + i + 1];
+              int s4[4];
+              s4[0] = (int)(s0 & 0xFFFFu) - (int)off * n_in_S;
+              s4[1] = (int)(s0 >> 16) - (int)off * n_in_S;
+              s4[2] = (int)(s1 & 0xFFFFu) - (int)off * n_in_S;
+              s4[3] = (int)(s1 >> 16) - (int)off * n_in_S;
+              if (n_merged > 0) {
+                s4[0] += (int)mv[2 * i]; s4[1] += (int)mv[2 * i + 1];
+                s4[2] += (int)mv[2 * i + 2]; s4[3] += (int)mv[2 * i + 3];
+              }
+              emit4<true>(p, gm, gn0 + c * 16 + 2 * i, s4, parked, vec, scale);
             }
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-    }
-    if (ok && gm < p.M) {
-      const float scale = (float)((double)__ldg(p.step_a) * (double)__ldg(p.step_b) *
-                                  (double)(1u << p.acc_shift) / (double)p.had_block);
-      float* orow = p.out + gm * p.ld_out;
-      const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
-                       (gn0 + 128 <= p.N);
-      if (vec) {
+    } else {
+      int S[EPI_COLS];
 #pragma unroll
-        for (int i = 0; i < 128; i += 4) {
-          float4 o;
-          o.x = __fmul_rn((float)S[i], scale);
-          o.y = __fmul_rn((float)S[i + 1], scale);
-          o.z = __fmul_rn((float)S[i + 2], scale);
-          o.w = __fmul_rn((float)S[i + 3], scale);
-          *reinterpret_cast<float4*>(orow + gn0 + i) = o;
-        }
-      } else {
+      for (int i = 0; i < EPI_COLS; ++i) S[i] = 0;
+      for (int ci = 0; ci < n_clamp_tiles; ++ci) {
+        const int buf = merging ? 1 : (ci & 1);
+        const uint32_t use = merging ? (uint32_t)ci : (uint32_t)(ci >> 1);
+        if (!mbar_wait_yield<32>(bar_tfull + 8 * buf, use & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
 #pragma unroll
-        for (int i = 0; i < 128; ++i) {
-          if (gn0 + i < p.N) orow[gn0 + i] = __fmul_rn((float)S[i], scale);
+        for (int c = 0; c < EPI_COLS / 16; ++c) {
+          uint32_t v[16];
+          HDQT_TMEM_LD16(lane_addr + buf * BN + c * 16, v);
+          HDQT_TMEM_WAIT16(v);
+          if (c == EPI_COLS / 16 - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int ct = acc_quant<kShift>((int)v[i], r, lo, hi);
+            S[c * 16 + i] += ct;
+            if (kTilesOut) {
+              const int64_t n = gn0 + c * 16 + i;
+              if (gm < p.M && n < p.N) {
+                const int64_t o = ((int64_t)ci * p.M + gm) * p.N + n;
+                if (p.tiles_elem_bytes == 1) reinterpret_cast<int8_t*>(p.tiles_out)[o] = (int8_t)ct;
+                else reinterpret_cast<int16_t*>(p.tiles_out)[o] = (int16_t)ct;
+              }
+            }
+          }
         }
       }
-      if (p.S_out != nullptr) {
-        int32_t* srow = p.S_out + gm * p.N;
+      if (ok && n_merged > 0) {
+        ok = mbar_wait_yield<1000>(bar_tfull + 0, 0u, abort_flag);
+        tc_fence_after();
+      }
+      if (ok) {
+        const float scale = (float)((double)__ldg(p.step_a) * (double)__ldg(p.step_b) *
+                                    (double)(1u << p.acc_shift) / (double)p.had_block);
 #pragma unroll
-        for (int i = 0; i < 128; ++i) {
-          if (gn0 + i < p.N) srow[gn0 + i] = S[i];
+        for (int c = 0; c < EPI_COLS / 16; ++c) {
+          uint32_t mv[16];
+          if (n_merged > 0) {   // uniform
+            HDQT_TMEM_LD16(lane_addr + c * 16, mv);
+            HDQT_TMEM_WAIT16(mv);
+          }
+          if (gm < p.M) {
+#pragma unroll
+            for (int i = 0; i < 16; i += 4) {
+              int s4[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                s4[j] = S[c * 16 + i + j];
+                if (n_merged > 0) s4[j] += (int)mv[i + j];
+              }
+              emit4<true>(p, gm, gn0 + c * 16 + i, s4, false, vec, scale);
+            }
+          }
         }
       }
     }
@@ -395,14 +740,15 @@ bool make_operand_map(CUtensorMap* map, const int8_t* base, int64_t rows, int64_
   return r == CUDA_SUCCESS;
 }
 
-template <bool kShift, bool kTilesOut>
+template <bool kPacked, bool kShift, bool kTilesOut>
 hdqt_status_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, dim3 grid,
                              cudaStream_t s) {
-  auto kern = gemm_i8_tiled_kernel<kShift, kTilesOut>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-    return HDQT_ERR_CUDA;
+  auto kern = gemm_i8_tiled_kernel<kPacked, kShift, kTilesOut>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (e != cudaSuccess) return cuda_failure(e, "cudaFuncSetAttribute(gemm)");
   kern<<<grid, GEMM_THREADS, SMEM_BYTES, s>>>(ma, mb, p);
-  return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
+  e = cudaGetLastError();
+  return e == cudaSuccess ? HDQT_OK : cuda_failure(e, "launch(gemm)");
 }
 
 }  // namespace
@@ -411,19 +757,20 @@ hdqt_status_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const
 
 using namespace hdqt;
 
-extern "C" size_t hdqt_gemm_i8_workspace_bytes(int64_t, int64_t, int64_t) { return 256; }
+extern "C" size_t hdqt_gemm_i8_workspace_bytes(int64_t, int64_t, int64_t) { return 16384; }
 
 extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, const float* step_a,
                                             const float* step_b, int64_t M, int64_t N, int64_t K_pad,
-                                            int32_t acc_bits, int32_t acc_tile, int32_t acc_shift,
-                                            int32_t had_block, float* out, int64_t ld_out, int32_t* S_out,
-                                            void* tiles_out, int32_t tiles_elem_bytes, const int32_t* norms_a,
-                                            const int32_t* norms_b, uint32_t flags, void* workspace,
-                                            size_t workspace_bytes, int32_t* dev_status, void* stream) {
-  (void)norms_a; (void)norms_b; (void)flags; (void)workspace;
+                                            int32_t code_bits, int32_t acc_bits, int32_t acc_tile,
+                                            int32_t acc_shift, int32_t had_block, float* out, int64_t ld_out,
+                                            int32_t* S_out, void* tiles_out, int32_t tiles_elem_bytes,
+                                            const int32_t* norms_a, const int32_t* norms_b, uint32_t flags,
+                                            void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                            void* stream) {
   if (!Aq || !Bq || !step_a || !step_b || !out) return HDQT_ERR_INVALID_ARG;
   if (M <= 0 || N <= 0 || K_pad <= 0 || ld_out < N) return HDQT_ERR_INVALID_ARG;
   if (K_pad % 32 != 0) return HDQT_ERR_INVALID_ARG;
+  if (code_bits < 2 || code_bits > 8) return HDQT_ERR_INVALID_ARG;
   if (acc_bits < 2 || acc_bits > 32 || acc_shift < 0 || acc_shift > 24) return HDQT_ERR_INVALID_ARG;
   if (acc_tile < 0 || acc_tile % 32 != 0) return HDQT_ERR_INVALID_ARG;
   if (had_block < 1 || (had_block & (had_block - 1)) != 0) return HDQT_ERR_INVALID_ARG;
@@ -436,20 +783,27 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
     else if (tiles_elem_bytes == 2) { if (acc_bits > 16) return HDQT_ERR_INVALID_ARG; }
     else return HDQT_ERR_INVALID_ARG;
   }
-  // the wide sum must fit int32: |c_t| <= 2^(b_a-1), T tiles
   const int64_t tiles32 = K_pad / 32;
   const int64_t tpa = acc_tile == 0 ? tiles32 : acc_tile / 32;
   const int64_t num_acc = (tiles32 + tpa - 1) / tpa;
-  const int64_t per_tile_max = acc_bits >= 32 ? (tpa * 32 * 128 * 128) : (int64_t(1) << (acc_bits - 1));
-  if (per_tile_max * num_acc > INT32_MAX || tpa * 32 * 128 * 128 > INT32_MAX) return HDQT_ERR_UNSUPPORTED;
+  // largest magnitude of one exact tile sum, given |code| <= 2^(code_bits-1)
+  const int64_t code_max = int64_t(1) << (code_bits - 1);
+  const int64_t p_max = tpa * 32 * code_max * code_max;
+  if (p_max > INT32_MAX) return HDQT_ERR_UNSUPPORTED;
+  // the wide sum must fit int32: |c_t| <= min(2^(b_a-1), p_max) per tile
+  const int64_t acc_max = acc_bits >= 32 ? p_max : (int64_t(1) << (acc_bits - 1));
+  const int64_t per_tile_max = acc_max < p_max ? acc_max : p_max;
+  if (per_tile_max * num_acc > INT32_MAX) return HDQT_ERR_UNSUPPORTED;
 
   CUtensorMap ma, mb;
   if (!make_operand_map(&ma, Aq, M, K_pad, BM) || !make_operand_map(&mb, Bq, N, K_pad, BN)) return HDQT_ERR_CUDA;
 
   GemmParams p;
+  memset(&p, 0, sizeof(p));
   p.M = M; p.N = N; p.K_pad = K_pad;
   p.tiles32 = (int32_t)tiles32;
   p.tiles_per_acc = (int32_t)tpa;
+  p.num_acc = (int32_t)num_acc;
   p.acc_shift = acc_shift;
   p.lo = acc_bits >= 32 ? INT32_MIN : -(1 << (acc_bits - 1));
   p.hi = acc_bits >= 32 ? INT32_MAX : (1 << (acc_bits - 1)) - 1;
@@ -458,14 +812,39 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
   p.out = out; p.ld_out = ld_out; p.S_out = S_out;
   p.tiles_out = tiles_out; p.tiles_elem_bytes = tiles_elem_bytes;
   p.dev_status = dev_status;
+  p.debug_mode = getenv("HDQT_GEMM_DEBUG") ? atoi(getenv("HDQT_GEMM_DEBUG")) : 0;
+  p.debug_ts = (p.debug_mode & 32) ? reinterpret_cast<long long*>(workspace) : nullptr;
+
+  // 16-bit-lane epilogue: tile sums fit int16, the offset sums fit uint16 for flush_every tiles
+  const bool packed = !tiles_out && acc_shift == 0 && acc_bits <= 8 && p_max <= 32767;
+  p.flush_every = packed ? (int32_t)(65535 / ((int64_t)p.hi - p.lo)) : 0;
+  if (p.flush_every > 256) p.flush_every = 256;
+
+  // merging of clamp-free tiles: only without rounding shift (the shift is not the identity)
+  p.merge = 0;
+  if (!tiles_out && acc_shift == 0 && !(flags & HDQT_FLAG_NO_MERGE)) {
+    if (p_max <= (int64_t)p.hi) {
+      p.merge = 2;  // no tile can clamp whatever the data
+    } else if (norms_a && norms_b && num_acc <= 32 * MAX_CERT_WORDS) {
+      p.merge = 1;
+      const int64_t thr = (int64_t)p.hi / tpa;
+      p.cert_thr_sq = thr * thr;
+      p.norms_a = norms_a;
+      p.norms_b = norms_b;
+      p.merge_max_uncert_256 = 32;  // merge in a CTA when at most 1/8 of its tiles need the clamp path
+    }
+  }
 
   const dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + BN - 1) / BN));
   if (grid.y > 65535) return HDQT_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (tiles_out) {
-    return acc_shift ? launch_variant<true, true>(ma, mb, p, grid, s) : launch_variant<false, true>(ma, mb, p, grid, s);
+    return acc_shift ? launch_variant<false, true, true>(ma, mb, p, grid, s)
+                     : launch_variant<false, false, true>(ma, mb, p, grid, s);
   }
-  return acc_shift ? launch_variant<true, false>(ma, mb, p, grid, s) : launch_variant<false, false>(ma, mb, p, grid, s);
+  if (packed) return launch_variant<true, false, false>(ma, mb, p, grid, s);
+  return acc_shift ? launch_variant<false, true, false>(ma, mb, p, grid, s)
+                   : launch_variant<false, false, false>(ma, mb, p, grid, s);
 }
 
 extern "C" hdqt_status_t hdqt_calibrate_acc_shift(const int8_t* Aq, const int8_t* Bq, int64_t M, int64_t N,

@@ -66,7 +66,7 @@ def _load() -> C.CDLL:
                                            vp, sz, vp, vp]
     lib.hdqt_quantize_workspace_bytes.argtypes = [i64, i64, i32]
     lib.hdqt_quantize_workspace_bytes.restype = sz
-    lib.hdqt_gemm_i8_tiled.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, vp, i64, vp, vp, i32,
+    lib.hdqt_gemm_i8_tiled.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp, i64, vp, vp, i32,
                                        vp, vp, u32, vp, sz, vp, vp]
     lib.hdqt_gemm_i8_workspace_bytes.argtypes = [i64, i64, i64]
     lib.hdqt_gemm_i8_workspace_bytes.restype = sz
@@ -173,7 +173,7 @@ def quantize_hadamard(src: torch.Tensor, had_block: int = 32, bits: int = 4, cli
 
 def gemm_i8_tiled(Aq: torch.Tensor, Bq: torch.Tensor, step_a: torch.Tensor, step_b: torch.Tensor,
                   acc_bits: int = 8, acc_tile: int = 32, acc_shift: int = 0, had_block: int = 32,
-                  want_S: bool = False, want_tiles: bool = False, norms_a=None, norms_b=None, flags: int = 0,
+                  code_bits: int = 4, want_S: bool = False, want_tiles: bool = False, norms_a=None, norms_b=None, flags: int = 0,
                   dev_status: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None):
     """Out[M,N] from codes Aq[M,K_pad], Bq[N,K_pad]. Returns (out, S or None, tiles or None)."""
     M, Kp = Aq.shape
@@ -194,7 +194,7 @@ def gemm_i8_tiled(Aq: torch.Tensor, Bq: torch.Tensor, step_a: torch.Tensor, step
         tiles = torch.empty((T, M, N), dtype=torch.int8 if elem == 1 else torch.int16, device=dev)
     ws = torch.empty(max(256, lib.hdqt_gemm_i8_workspace_bytes(M, N, Kp)), dtype=torch.uint8, device=dev)
     _check(lib.hdqt_gemm_i8_tiled(Aq.data_ptr(), Bq.data_ptr(), step_a.data_ptr(), step_b.data_ptr(), M, N, Kp,
-                                  acc_bits, acc_tile, acc_shift, had_block, out.data_ptr(), out.stride(0),
+                                  code_bits, acc_bits, acc_tile, acc_shift, had_block, out.data_ptr(), out.stride(0),
                                   _ptr(S), _ptr(tiles), elem, _ptr(norms_a), _ptr(norms_b), flags, ws.data_ptr(),
                                   ws.numel(), _ptr(dev_status), _stream()), "hdqt_gemm_i8_tiled")
     return out, S, tiles

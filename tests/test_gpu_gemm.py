@@ -92,7 +92,7 @@ def test_i8_tiled_saturating_and_8bit_codes(hdqt):
     rng = np.random.default_rng(3)
     A8, B8 = _codes(rng, 64, 128, -128, 128), _codes(rng, 48, 128, -128, 128)
     _, want_S, _ = O.gemm_i8_tiled(A8, B8, 1.0, 1.0, 32, 0, 0, 32)
-    _, S, _ = hdqt.gemm_i8_tiled(_dev(A8), _dev(B8), one, one, 32, 0, 0, 32, want_S=True)
+    _, S, _ = hdqt.gemm_i8_tiled(_dev(A8), _dev(B8), one, one, 32, 0, 0, 32, code_bits=8, want_S=True)
     assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
 
 
@@ -150,7 +150,13 @@ def _run_three(hdqt, X, W, G, w_is_cd=False, **over):
         # integer sums: re-run the integer GEMM on the codes the library produced
         _, S, tiles = hdqt.gemm_i8_tiled(ws.codes_a(), ws.codes_b(), ws.scalar("step_a"), ws.scalar("step_b"),
                                          desc.acc_bits, desc.acc_tile, desc.acc_shift, desc.had_block,
-                                         want_S=True, want_tiles=desc.acc_bits <= 16)
+                                         code_bits=desc.in_bits, want_S=True, want_tiles=desc.acc_bits <= 16)
+        # the production variants (no per-tile debug output; with and without clamp-free tile merging)
+        for flags in (0, hdqt.FLAG_NO_MERGE):
+            _, S2, _ = hdqt.gemm_i8_tiled(ws.codes_a(), ws.codes_b(), ws.scalar("step_a"), ws.scalar("step_b"),
+                                          desc.acc_bits, desc.acc_tile, desc.acc_shift, desc.had_block,
+                                          code_bits=desc.in_bits, want_S=True, flags=flags)
+            assert torch.equal(S2, S), (kind, flags)
         want_S = want["S"].T if swapped else want["S"]
         assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), kind
         if tiles is not None:
@@ -225,3 +231,84 @@ def test_sampled_parity_at_sweep_size(hdqt):
     _assert_close(got[rows], want_rows)
     _assert_close(got[:, cols], want_cols)
     assert np.array_equal(got[rows], want_rows) and np.array_equal(got[:, cols], want_cols)
+
+
+# ---- clamp-free tile merging and the 16-bit-lane epilogue --------------------------------------------
+
+def _tile_norms(codes):
+    rows, Kp = codes.shape
+    sq = (codes.astype(np.int64) ** 2).reshape(rows, Kp // 32, 32).sum(2)
+    nb = (rows + 127) // 128
+    return np.stack([sq[b * 128:(b + 1) * 128].max(0) for b in range(nb)]).astype(np.int32)
+
+
+def _sparse_codes(rng, rows, K, density):
+    c = rng.integers(-8, 8, size=(rows, K))
+    return (c * (rng.random((rows, K)) < density)).astype(np.int8)
+
+
+@pytest.mark.parametrize("density_a,density_b", [(0.05, 0.05), (0.3, 0.1), (1.0, 0.02), (1.0, 1.0)])
+@pytest.mark.parametrize("acc_bits,acc_tile", [(8, 32), (8, 64), (6, 32)])
+def test_merging_is_bit_identical(hdqt, density_a, density_b, acc_bits, acc_tile):
+    """Mixed certified / uncertified tiles: merged, unmerged and oracle sums agree exactly."""
+    rng = np.random.default_rng(int(density_a * 100) * 7 + int(density_b * 100) + acc_bits + acc_tile)
+    M, N, K = 200, 300, 1024
+    Aq, Bq = _sparse_codes(rng, M, K, density_a), _sparse_codes(rng, N, K, density_b)
+    # make certification vary along K: a dense stripe of tiles
+    Aq[:, 256:384] = rng.integers(-8, 8, size=(M, 128))
+    Bq[:, 320:448] = rng.integers(-8, 8, size=(N, 128))
+    _, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 1.0, 1.0, acc_bits, acc_tile, 0, 32)
+    one = torch.ones(1, device="cuda")
+    na, nb = _dev(_tile_norms(Aq)), _dev(_tile_norms(Bq))
+    status = hdqt.new_status("cuda")
+    for flags in (0, hdqt.FLAG_NO_MERGE):
+        _, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), one, one, acc_bits, acc_tile, 0, 32, want_S=True,
+                                     norms_a=na, norms_b=nb, flags=flags, dev_status=status)
+        hdqt.check_device_status(status)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), flags
+
+
+def test_merging_with_norms_from_the_quantizer(hdqt):
+    """Heavy-tailed operands: most tiles certify; the composite call (merging on) equals the oracle."""
+    A = inputs.heavy_tailed(300, 2048, seed=21)
+    B = inputs.heavy_tailed(520, 2048, seed=22)
+    want = O.gemm_dgrad(A, B, O.dgrad_desc(seed=3, tag_a=2, tag_b=3))
+    status = hdqt.new_status("cuda")
+    out, ws = hdqt.gemm_dgrad(_dev(A), _dev(B), desc=hdqt.default_desc("dgrad", seed=3), dev_status=status)
+    hdqt.check_device_status(status)
+    assert np.array_equal(out.cpu().numpy(), want["out"])
+    out2, _ = hdqt.gemm_dgrad(_dev(A), _dev(B), desc=hdqt.default_desc("dgrad", seed=3, flags=hdqt.FLAG_NO_MERGE))
+    assert torch.equal(out, out2)
+    # the certified fraction is what makes merging worthwhile on such data: check it is large
+    na = _tile_norms(want["Aq"]).astype(np.int64)
+    nb = _tile_norms(want["Bq"]).astype(np.int64)
+    nb256 = np.stack([nb[2 * j:2 * j + 2].max(0) for j in range((nb.shape[0] + 1) // 2)])
+    cert = (na[:, None, :] * nb256[None, :, :]) <= 127 * 127
+    assert cert.mean() > 0.9
+
+
+def test_long_contraction_widens_packed_sums(hdqt):
+    """More than 256 clamp tiles: the 16-bit lane sums are widened through the output buffer."""
+    rng = np.random.default_rng(31)
+    M, N, K = 130, 70, 32 * 700
+    Aq, Bq = _codes(rng, M, K), _codes(rng, N, K)
+    Aq[:, :] = np.where(rng.random((M, K)) < 0.5, 7, Aq)       # push many tiles into saturation
+    want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 0.5, 0.125)
+    half, eighth = torch.tensor([0.5], device="cuda"), torch.tensor([0.125], device="cuda")
+    # odd leading dimension: exercises the scalar store path of the widening too
+    big = torch.zeros((M, N + 3), device="cuda")
+    for view in (None, big[:, 1:N + 1]):
+        out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), half, eighth, want_S=True, out=view)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
+        assert np.array_equal(out.cpu().numpy(), want_out)
+
+
+def test_wide_accumulators_merge_without_norms(hdqt):
+    """b_a >= 13 with 4-bit codes: no tile can clamp, every tile is merged; equals the plain int matmul."""
+    rng = np.random.default_rng(32)
+    Aq, Bq = _codes(rng, 150, 480), _codes(rng, 260, 480)
+    plain = Aq.astype(np.int64) @ Bq.astype(np.int64).T
+    one = torch.ones(1, device="cuda")
+    for acc_bits in (13, 16, 32):
+        _, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), one, one, acc_bits, 32, 0, 32, want_S=True)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), plain)

@@ -110,6 +110,8 @@ def test_sr_bits_layout_and_uniformity():
     for word in w:
         want += [int(word[0]) & 0xFFFF, int(word[0]) >> 16]
     assert list(u[8 * g:8 * g + 8]) == want
+    # the whole-tensor form draws the same bits as the per-index form
+    assert np.array_equal(O.sr_random_u16_tensor(123, 5, 64, 512).ravel(), u)
     # chi-square over 16 equal bins: 15 dof, 99.99 % quantile ~ 44.3
     counts = np.bincount(u >> 12, minlength=16)
     chi2 = ((counts - len(u) / 16) ** 2 / (len(u) / 16)).sum()
