@@ -64,8 +64,6 @@ struct GemmParams {
   void* tiles_out;
   int32_t tiles_elem_bytes;
   int32_t* dev_status;
-  int32_t debug_mode;
-  long long* debug_ts;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -391,7 +389,6 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const int s = kb % STAGES;
         const uint32_t par = ((kb / STAGES) & 1) ^ 1;
         if (!mbar_wait(bar_empty + 8 * s, par, abort_flag)) break;
-        if (p.debug_mode & 2) { mbar_arrive(bar_full + 8 * s); issued = kb + 1; continue; }
         mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
         const uint32_t a_dst = smem_base + s * STAGE_BYTES;
         tma_load_2d(a_dst, &map_a, kb * BKB, m0, bar_full + 8 * s);
@@ -524,35 +521,29 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       uint32_t v0[EPI_COLS / 4], v1[EPI_COLS / 4];
       if (n_clamp_tiles > 0) {
         const int buf = merging ? 1 : 0;
-        if (!mbar_wait_yield<32>(bar_tfull + 8 * buf, 0u, abort_flag)) ok = false;
+        if (!mbar_wait(bar_tfull + 8 * buf, 0u, abort_flag)) ok = false;
         tc_fence_after();
         if (ok) HDQT_TMEM_LD16_PACK16(lane_addr + buf * BN, v0);
       }
       for (int ci = 0; ci < n_clamp_tiles && ok; ++ci) {
         const int buf = merging ? 1 : (ci & 1);
-        if (!(p.debug_mode & 8)) HDQT_TMEM_WAIT16(v0);                                         // first half of tile ci has landed
-        if (!(p.debug_mode & 8)) HDQT_TMEM_LD16_PACK16(lane_addr + buf * BN + EPI_COLS / 2, v1);  // second half in flight ...
-        if (!(p.debug_mode & 4)) {
+        HDQT_TMEM_WAIT16(v0);                                            // first half of tile ci has landed
+        HDQT_TMEM_LD16_PACK16(lane_addr + buf * BN + EPI_COLS / 2, v1);  // second half in flight ...
 #pragma unroll
         for (int i = 0; i < EPI_COLS / 4; ++i) S[i] += __viaddmin_s16x2_relu(v0[i], off2, rng2);
-        }
-        if (!(p.debug_mode & 8)) HDQT_TMEM_WAIT16(v1);                                         // ... landed: the buffer is free
+        HDQT_TMEM_WAIT16(v1);                                            // ... landed: the buffer is free
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-        if (p.debug_ts && blockIdx.x == 0 && blockIdx.y == 0 && warp == 2 && lane == 0 && ci >= 32 && ci < 96) p.debug_ts[(ci - 32) * 4 + 3] = clock64();
         if (ci + 1 < n_clamp_tiles) {
           const int nbuf = merging ? 1 : ((ci + 1) & 1);
           const uint32_t use = merging ? (uint32_t)(ci + 1) : (uint32_t)((ci + 1) >> 1);
-          if (!mbar_wait_yield<32>(bar_tfull + 8 * nbuf, use & 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar_tfull + 8 * nbuf, use & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          if (p.debug_ts && blockIdx.x == 0 && blockIdx.y == 0 && warp == 2 && lane == 0 && ci + 1 >= 32 && ci + 1 < 96) p.debug_ts[(ci + 1 - 32) * 4 + 2] = clock64();
-          if (!(p.debug_mode & 8)) HDQT_TMEM_LD16_PACK16(lane_addr + nbuf * BN, v0);           // first half of the next tile in flight
+          HDQT_TMEM_LD16_PACK16(lane_addr + nbuf * BN, v0);              // first half of the next tile in flight
         }
-        if (!(p.debug_mode & 4)) {
 #pragma unroll
         for (int i = 0; i < EPI_COLS / 4; ++i) S[EPI_COLS / 4 + i] += __viaddmin_s16x2_relu(v1[i], off2, rng2);
-        }
         if (++n_in_S == p.flush_every && ci + 1 < n_clamp_tiles) {
           // widen: park int32 partial sums in the output buffer
           if (gm < p.M) {
@@ -611,7 +602,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       for (int ci = 0; ci < n_clamp_tiles; ++ci) {
         const int buf = merging ? 1 : (ci & 1);
         const uint32_t use = merging ? (uint32_t)ci : (uint32_t)(ci >> 1);
-        if (!mbar_wait_yield<32>(bar_tfull + 8 * buf, use & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar_tfull + 8 * buf, use & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < EPI_COLS / 16; ++c) {
@@ -757,7 +748,7 @@ hdqt_status_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const
 
 using namespace hdqt;
 
-extern "C" size_t hdqt_gemm_i8_workspace_bytes(int64_t, int64_t, int64_t) { return 16384; }
+extern "C" size_t hdqt_gemm_i8_workspace_bytes(int64_t, int64_t, int64_t) { return 256; }
 
 extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, const float* step_a,
                                             const float* step_b, int64_t M, int64_t N, int64_t K_pad,
@@ -767,6 +758,7 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
                                             const int32_t* norms_a, const int32_t* norms_b, uint32_t flags,
                                             void* workspace, size_t workspace_bytes, int32_t* dev_status,
                                             void* stream) {
+  (void)workspace;
   if (!Aq || !Bq || !step_a || !step_b || !out) return HDQT_ERR_INVALID_ARG;
   if (M <= 0 || N <= 0 || K_pad <= 0 || ld_out < N) return HDQT_ERR_INVALID_ARG;
   if (K_pad % 32 != 0) return HDQT_ERR_INVALID_ARG;
@@ -812,8 +804,6 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
   p.out = out; p.ld_out = ld_out; p.S_out = S_out;
   p.tiles_out = tiles_out; p.tiles_elem_bytes = tiles_elem_bytes;
   p.dev_status = dev_status;
-  p.debug_mode = getenv("HDQT_GEMM_DEBUG") ? atoi(getenv("HDQT_GEMM_DEBUG")) : 0;
-  p.debug_ts = (p.debug_mode & 32) ? reinterpret_cast<long long*>(workspace) : nullptr;
 
   // 16-bit-lane epilogue: tile sums fit int16, the offset sums fit uint16 for flush_every tiles
   const bool packed = !tiles_out && acc_shift == 0 && acc_bits <= 8 && p_max <= 32767;
