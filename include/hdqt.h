@@ -58,7 +58,8 @@ typedef enum {
   HDQT_ERR_WORKSPACE = 4,    /* workspace smaller than hdqt_*_workspace_bytes  */
   HDQT_ERR_NONFINITE = 5,    /* (device) NaN/Inf in a transformed operand      */
   HDQT_ERR_TIMEOUT = 6,      /* (device) a bounded wait inside a kernel ran out*/
-  HDQT_ERR_CUDA = 7          /* a CUDA runtime / driver call failed            */
+  HDQT_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed            */
+  HDQT_ERR_STATIC_SCRATCH = 8 /* operand too large for the library's built-in scratch array */
 } hdqt_status_t;
 
 typedef enum {
@@ -149,6 +150,42 @@ hdqt_status_t hdqt_quantize_hadamard(const float* src, int64_t rows, int64_t K,
                                      int32_t* dev_status, void* stream);
 
 size_t hdqt_quantize_workspace_bytes(int64_t rows, int64_t K, int32_t had_block);
+
+/*
+ * hdqt_quantize_hadamard for callers that must not allocate device memory.
+ * (The paper has no counterpart: this is a deployment convenience, not part of the method.)
+ *
+ * Some callers cannot provide the workspace the call above needs, because they are not allowed
+ * to call cudaMalloc (or any allocating library routine) at the point where they quantize: code
+ * that runs after the application has handed all device memory to its own pool, plug-ins whose
+ * host forbids allocation, or latency-critical loops that cannot afford the device-wide
+ * synchronisation an allocation implies.  For them this entry point computes exactly what
+ * hdqt_quantize_hadamard computes with amax_in == NULL (same codes, step and tile norms, bit for
+ * bit) but takes its scratch from a fixed device array built into the library, so the call performs
+ * no cudaMalloc / cudaFree and needs no workspace argument.  Inputs and outputs are still the
+ * caller's buffers.
+ *
+ * Limits and rules
+ *   - The array is HDQT_STATIC_SCRATCH_BYTES (4 MiB + 256 B) and exists once per GPU for as long
+ *     as the library stays loaded.  It must hold 2 bytes per (row, 32-wide K tile):
+ *     rows * (K_pad / 32) <= 2 097 152 (e.g. 8192 x 8192).  Larger operands are refused with
+ *     HDQT_ERR_STATIC_SCRATCH and nothing is launched; use hdqt_quantize_hadamard then.
+ *   - The first call on each device looks up the array's device address (a cheap runtime query,
+ *     made with that device current); make that first call during set-up, before any stream
+ *     capture you may do.
+ *   - All calls on a device share the one array, and it keeps what the previous call left in it.
+ *     Each call re-initialises the parts that must start from zero, so back-to-back calls on one
+ *     stream are fine; calls that can overlap on the GPU (different streams, no ordering between
+ *     them) race on the array and corrupt each other's results.
+ */
+#define HDQT_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u + 256u)
+
+hdqt_status_t hdqt_quantize_hadamard_static(const float* src, int64_t rows, int64_t K,
+                                            int64_t ld_row, int64_t ld_k, int32_t had_block,
+                                            int32_t bits, float clip, int32_t mode,
+                                            uint64_t seed, uint32_t tag, int8_t* codes,
+                                            float* step_out, int32_t* tile_norms,
+                                            int32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------ */
 /* Tiled integer GEMM with low-bit tile accumulators (Section 3, last para.)  */

@@ -39,6 +39,7 @@ extern "C" const char* hdqt_status_string(hdqt_status_t s) {
     case HDQT_ERR_NONFINITE: return "non-finite value in an operand";
     case HDQT_ERR_TIMEOUT: return "bounded device wait ran out";
     case HDQT_ERR_CUDA: return "CUDA call failed";
+    case HDQT_ERR_STATIC_SCRATCH: return "operand too large for the built-in scratch array";
   }
   return "unknown status";
 }

@@ -13,6 +13,8 @@
 // Both are HBM-bound streaming kernels: 4 B/element read (+1 B/element written when
 // quantizing).  Butterfly order is ascending stride, every add/sub is a single fp32 rounding,
 // so the transformed values - and hence the codes - are bit-identical for both layouts.
+#include <mutex>
+
 #include "hdqt_common.cuh"
 
 namespace hdqt {
@@ -446,3 +448,68 @@ hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t
 }
 
 }  // namespace hdqt
+
+// ---- allocation-free variant of the transform + quantize call ----------------------------------
+//
+// Scratch for hdqt_quantize_hadamard_static lives in this fixed device array instead of a caller
+// workspace: [0, 256) holds the calibration maximum, the rest holds the per-row tile norms.
+// Every GPU that loads the library carries these HDQT_STATIC_SCRATCH_BYTES until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[HDQT_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_scratch_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+
+// In host code the name g_static_scratch is only a handle for the runtime, not a device address;
+// the address a kernel can use must be asked for, once per device, with that device current.
+hdqt_status_t static_scratch_for_current_device(unsigned char** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return hdqt::cuda_failure(e, "cudaGetDevice(static scratch)");
+  if (dev < 0 || dev >= kMaxDevices) return HDQT_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess || ptr == nullptr) return hdqt::cuda_failure(e, "cudaGetSymbolAddress(static scratch)");
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  *out = static_cast<unsigned char*>(g_static_scratch_ptr[dev]);
+  return HDQT_OK;
+}
+
+}  // namespace
+
+extern "C" hdqt_status_t hdqt_quantize_hadamard_static(const float* src, int64_t rows, int64_t K, int64_t ld_row,
+                                                       int64_t ld_k, int32_t had_block, int32_t bits, float clip,
+                                                       int32_t mode, uint64_t seed, uint32_t tag, int8_t* codes,
+                                                       float* step_out, int32_t* tile_norms, int32_t* dev_status,
+                                                       void* stream) {
+  // same argument rules as hdqt_quantize_hadamard
+  if (!src || !codes || !step_out || rows <= 0 || K <= 0) return HDQT_ERR_INVALID_ARG;
+  if (had_block < 1 || (had_block & (had_block - 1)) != 0) return HDQT_ERR_INVALID_ARG;
+  if (had_block > 32) return HDQT_ERR_UNSUPPORTED;
+  if (!((ld_k == 1 && ld_row >= K) || (ld_row == 1 && ld_k >= rows))) return HDQT_ERR_INVALID_ARG;
+  if (bits < 2 || bits > 8) return HDQT_ERR_INVALID_ARG;
+  if (!(clip >= 1.0f / 64.0f && clip <= 1.0f)) return HDQT_ERR_INVALID_ARG;
+  if (mode != HDQT_ROUND_NEAREST && mode != HDQT_ROUND_STOCHASTIC) return HDQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(src) & 3) || (reinterpret_cast<uintptr_t>(codes) & 127)) return HDQT_ERR_ALIGNMENT;
+  // the fixed array bounds the operand: 256 bytes + 2 bytes per (row, 32-wide K tile)
+  const int64_t tiles = hdqt_padded_k(K, had_block) / 32;
+  if (rows > (int64_t)(HDQT_STATIC_SCRATCH_BYTES - 256) / 2 / tiles) return HDQT_ERR_STATIC_SCRATCH;
+
+  unsigned char* scratch = nullptr;
+  hdqt_status_t st = static_scratch_for_current_device(&scratch);
+  if (st != HDQT_OK) return st;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  float* amax = reinterpret_cast<float*>(scratch);
+  uint16_t* row_norms = reinterpret_cast<uint16_t*>(scratch + 256);
+  // the array keeps whatever the previous call left: launch_absmax zeroes the maximum before it
+  // accumulates into it, and every row-norm entry that is read is written first by this call
+  st = hdqt::launch_absmax(src, rows, K, ld_row, ld_k, had_block, amax, dev_status, s);
+  if (st != HDQT_OK) return st;
+  return hdqt::launch_quantize(src, rows, K, ld_row, ld_k, had_block, bits, clip, mode, seed, tag, amax, codes,
+                               step_out, tile_norms, row_norms, dev_status, s);
+}

@@ -24,7 +24,7 @@ EXPORTED = [
     "hdqt_default_desc", "hdqt_padded_k", "hdqt_status_string", "hdqt_absmax_hadamard",
     "hdqt_quantize_hadamard", "hdqt_quantize_workspace_bytes", "hdqt_gemm_i8_tiled",
     "hdqt_gemm_i8_workspace_bytes", "hdqt_calibrate_acc_shift", "hdqt_gemm_fwd", "hdqt_gemm_dgrad",
-    "hdqt_gemm_wgrad", "hdqt_workspace_bytes", "hdqt_workspace_layout",
+    "hdqt_gemm_wgrad", "hdqt_workspace_bytes", "hdqt_workspace_layout", "hdqt_quantize_hadamard_static",
 ]
 
 
@@ -64,6 +64,9 @@ def _load() -> C.CDLL:
     lib.hdqt_absmax_hadamard.argtypes = [vp, i64, i64, i64, i64, i32, vp, vp, vp]
     lib.hdqt_quantize_hadamard.argtypes = [vp, i64, i64, i64, i64, i32, i32, f32, i32, u64, u32, vp, vp, vp, vp,
                                            vp, sz, vp, vp]
+    lib.hdqt_quantize_hadamard_static.argtypes = [vp, i64, i64, i64, i64, i32, i32, f32, i32, u64, u32, vp, vp, vp,
+                                                  vp, vp]
+    lib.hdqt_quantize_hadamard_static.restype = C.c_int
     lib.hdqt_quantize_workspace_bytes.argtypes = [i64, i64, i32]
     lib.hdqt_quantize_workspace_bytes.restype = sz
     lib.hdqt_gemm_i8_tiled.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp, i64, vp, vp, i32,
@@ -168,6 +171,25 @@ def quantize_hadamard(src: torch.Tensor, had_block: int = 32, bits: int = 4, cli
     _check(lib.hdqt_quantize_hadamard(src.data_ptr(), rows, K, ld_row, ld_k, had_block, bits, clip, mode, seed, tag,
                                       _ptr(amax), codes.data_ptr(), step.data_ptr(), _ptr(norms), ws.data_ptr(),
                                       ws.numel(), _ptr(dev_status), _stream()), "hdqt_quantize_hadamard")
+    return codes, step, norms
+
+
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 + 256
+
+
+def quantize_hadamard_static(src: torch.Tensor, codes: torch.Tensor, step: torch.Tensor,
+                             norms: Optional[torch.Tensor] = None, had_block: int = 32, bits: int = 4,
+                             clip: float = 1.0, mode: int = ROUND_NEAREST, seed: int = 0, tag: int = 0,
+                             dev_status: Optional[torch.Tensor] = None):
+    """Same result as quantize_hadamard (measured maximum), written into buffers the caller already
+    owns, for callers that cannot allocate device memory at this point: the library's built-in
+    scratch array replaces the workspace, so neither this wrapper nor the C call allocates anything.
+    Operands are limited to rows * K_pad / 32 <= 2 097 152; calls on different streams must not
+    overlap (they share the one array)."""
+    rows, K, ld_row, ld_k = _view_2d(src)
+    _check(lib.hdqt_quantize_hadamard_static(src.data_ptr(), rows, K, ld_row, ld_k, had_block, bits, clip, mode,
+                                             seed, tag, codes.data_ptr(), step.data_ptr(), _ptr(norms),
+                                             _ptr(dev_status), _stream()), "hdqt_quantize_hadamard_static")
     return codes, step, norms
 
 
