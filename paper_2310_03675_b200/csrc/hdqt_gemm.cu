@@ -35,6 +35,9 @@ constexpr int EPI_COLS = BN / (NUM_EPI_WARPS / 4);
 constexpr int GEMM_THREADS = 32 * (2 + NUM_EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int MAX_CERT_WORDS = 512;            // certificate bitmask: up to 16384 accumulator tiles
+constexpr int STAGE_OUT_ROW = EPI_COLS + 4;     // floats per staged output row (+4: conflict-free float4 rows)
+constexpr int STAGE_OUT_WARP = 32 * STAGE_OUT_ROW;   // floats per epilogue warp (32 rows x 64 columns)
+static_assert(NUM_EPI_WARPS * STAGE_OUT_WARP * 4 <= STAGES * STAGE_BYTES, "output staging must fit the operand ring");
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 4 * MAX_CERT_WORDS;
 
 // instruction descriptor: D = s32, A = B = signed 8-bit, both K-major, N = 256, M = 128
@@ -246,9 +249,12 @@ __device__ __forceinline__ int acc_quant(int P, int r, int lo, int hi) {
 // Writes 4 consecutive output columns of one row: the final fp32 values (and optionally the integer
 // sums), or - for an intermediate widening of the packed sums - the int32 partial sums, which are
 // parked in the output buffer itself until the final pass reads them back.
+// In the final pass of the vector path the fp32 values go to `stage` (this thread's row of the warp's
+// shared-memory staging block) instead, and the warp copies the block out row by row afterwards, so
+// that global stores are 256 contiguous bytes per half-warp rather than 16 bytes per row.
 template <bool kFinal>
 __device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t gn, int (&s)[4], bool have_prev,
-                                      bool vec, float scale) {
+                                      bool vec, float scale, float* stage = nullptr) {
   float* orow = p.out + gm * p.ld_out + gn;
   if (vec) {
     if (have_prev) {
@@ -261,7 +267,7 @@ __device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t g
       o.y = __fmul_rn((float)s[1], scale);
       o.z = __fmul_rn((float)s[2], scale);
       o.w = __fmul_rn((float)s[3], scale);
-      *reinterpret_cast<float4*>(orow) = o;
+      *reinterpret_cast<float4*>(stage != nullptr ? stage : orow) = o;
     } else {
       *reinterpret_cast<int4*>(orow) = make_int4(s[0], s[1], s[2], s[3]);
     }
@@ -308,8 +314,23 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * BM;
-  const int n0 = blockIdx.y * BN;
+  // 1-D grid over output blocks, ordered so that co-resident CTAs form a roughly square patch
+  // (16 row blocks x ~9 column blocks on 148 SMs): both operands' panels are then shared through L2
+  const int tiles_m = (int)((p.M + BM - 1) / BM), tiles_n = (int)((p.N + BN - 1) / BN);
+  int tile_m, tile_n;
+  {
+    constexpr int GROUP_M = 16;
+    const int t = blockIdx.x;
+    const int per_group = GROUP_M * tiles_n;
+    const int group = t / per_group;
+    const int first_m = group * GROUP_M;
+    const int group_rows = min(tiles_m - first_m, GROUP_M);
+    const int in_group = t - group * per_group;
+    tile_m = first_m + in_group % group_rows;
+    tile_n = in_group / group_rows;
+  }
+  const int m0 = tile_m * BM;
+  const int n0 = tile_n * BN;
   const int num_kblocks = (p.tiles32 + 3) >> 2;
   const int num_acc = p.num_acc;
 
@@ -345,8 +366,8 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     if (warp >= 2) {
       const int et = threadIdx.x - 64;
       const int64_t T = p.tiles32;
-      const int32_t* na = p.norms_a + (int64_t)blockIdx.x * T;
-      const int64_t nb_blk = (int64_t)blockIdx.y * 2;
+      const int32_t* na = p.norms_a + (int64_t)tile_m * T;
+      const int64_t nb_blk = (int64_t)tile_n * 2;
       const int32_t* nb0 = p.norms_b + nb_blk * T;
       const bool has1 = (nb_blk + 1) * 128 < p.N;
       const int32_t* nb1 = nb0 + T;
@@ -505,6 +526,23 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
                      (gn0 + EPI_COLS <= p.N);
     bool ok = true;
+    // output staging reuses the operand ring: it is touched only after the last MMA has completed
+    float* stage_warp = reinterpret_cast<float*>(smem_al) + (warp - 2) * STAGE_OUT_WARP;
+    float* stage_row = stage_warp + lane * STAGE_OUT_ROW;
+    // copies the warp's staged 32 x 64 block to global memory, two rows (2 x 256 bytes) per instruction
+    auto copy_out = [&]() {
+      __syncwarp();
+      const int sub_row = lane >> 4, c4 = (lane & 15) * 4;
+#pragma unroll 4
+      for (int rr = 0; rr < 32; rr += 2) {
+        const int rloc = rr + sub_row;
+        const int64_t grow = (int64_t)m0 + q * 32 + rloc;
+        if (grow < p.M) {
+          const float4 v = *reinterpret_cast<const float4*>(stage_warp + rloc * STAGE_OUT_ROW + c4);
+          *reinterpret_cast<float4*>(p.out + grow * p.ld_out + gn0 + c4) = v;
+        }
+      }
+    };
 
     if (kPacked) {
       // two columns per register: low half = even column, high half = odd column
@@ -564,7 +602,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
       }
       if (ok && n_merged > 0) {
-        ok = mbar_wait_yield<1000>(bar_tfull + 0, 0u, abort_flag);
+        ok = mbar_wait_yield<256>(bar_tfull + 0, 0u, abort_flag);
         tc_fence_after();
       }
       if (ok) {
@@ -590,10 +628,12 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 s4[0] += (int)mv[2 * i]; s4[1] += (int)mv[2 * i + 1];
                 s4[2] += (int)mv[2 * i + 2]; s4[3] += (int)mv[2 * i + 3];
               }
-              emit4<true>(p, gm, gn0 + c * 16 + 2 * i, s4, parked, vec, scale);
+              emit4<true>(p, gm, gn0 + c * 16 + 2 * i, s4, parked, vec, scale,
+                          vec ? stage_row + c * 16 + 2 * i : nullptr);
             }
           }
         }
+        if (vec) copy_out();
       }
     } else {
       int S[EPI_COLS];
@@ -630,7 +670,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
       }
       if (ok && n_merged > 0) {
-        ok = mbar_wait_yield<1000>(bar_tfull + 0, 0u, abort_flag);
+        ok = mbar_wait_yield<256>(bar_tfull + 0, 0u, abort_flag);
         tc_fence_after();
       }
       if (ok) {
@@ -652,10 +692,11 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 s4[j] = S[c * 16 + i + j];
                 if (n_merged > 0) s4[j] += (int)mv[i + j];
               }
-              emit4<true>(p, gm, gn0 + c * 16 + i, s4, false, vec, scale);
+              emit4<true>(p, gm, gn0 + c * 16 + i, s4, false, vec, scale, vec ? stage_row + c * 16 + i : nullptr);
             }
           }
         }
+        if (vec) copy_out();
       }
     }
   }
@@ -825,8 +866,9 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
     }
   }
 
-  const dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + BN - 1) / BN));
-  if (grid.y > 65535) return HDQT_ERR_UNSUPPORTED;
+  const int64_t num_blocks = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+  if (num_blocks > INT32_MAX) return HDQT_ERR_UNSUPPORTED;
+  const dim3 grid((unsigned)num_blocks);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (tiles_out) {
     return acc_shift ? launch_variant<false, true, true>(ma, mb, p, grid, s)

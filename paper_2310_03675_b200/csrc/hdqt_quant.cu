@@ -57,22 +57,24 @@ __device__ __forceinline__ void fwht8_regs(float (&x)[8], int had_block) {
   }
 }
 
-// strides 8 and 16 across lanes (lane^1, lane^2); the whole warp must call this
+// strides 8 and 16 across lanes (lane^1, lane^2); the whole warp must call this.
+// The lower lane of a pair needs x + y, the upper one y - x: both are fma(sign, x, y) with sign = +-1
+// (sign*x is exact, so the fused form rounds once, exactly like the add / subtract).
 __device__ __forceinline__ void fwht8_lanes(float (&x)[8], int had_block, int lane) {
   if (had_block > 8) {
-    const bool upper = lane & 1;
+    const float sign = (lane & 1) ? -1.0f : 1.0f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float y = __shfl_xor_sync(0xFFFFFFFFu, x[i], 1);
-      x[i] = upper ? __fsub_rn(y, x[i]) : __fadd_rn(x[i], y);
+      x[i] = __fmaf_rn(sign, x[i], y);
     }
   }
   if (had_block > 16) {
-    const bool upper = lane & 2;
+    const float sign = (lane & 2) ? -1.0f : 1.0f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float y = __shfl_xor_sync(0xFFFFFFFFu, x[i], 2);
-      x[i] = upper ? __fsub_rn(y, x[i]) : __fadd_rn(x[i], y);
+      x[i] = __fmaf_rn(sign, x[i], y);
     }
   }
 }
@@ -190,30 +192,65 @@ __device__ __forceinline__ void block_absmax_commit(uint32_t mx, float* amax_out
 }
 
 // ---- K-contiguous kernels -------------------------------------------------------------------
+// A thread block walks the tensor in slabs of kUnroll*kThreads chunks (a chunk = 8 consecutive k of one
+// row); every thread first issues the loads of its kUnroll chunks, then transforms them, so that
+// kUnroll*32 bytes per thread are in flight.
+
+constexpr int kUnrollAbsmax = 4;
+constexpr int kUnrollQuant = 2;
+
+// chunk index -> (row, first k). 64-bit division is ~100 instructions, i.e. more than the whole
+// transform of the chunk, so it is kept for huge tensors only.
+struct ChunkMap {
+  int64_t chunks_per_row;
+  bool small;   // every chunk index fits 32 bits
+};
+__device__ __forceinline__ void chunk_to_row_k(const ChunkMap& m, int64_t c, int64_t& r, int64_t& k0) {
+  if (m.small) {
+    const uint32_t rr = (uint32_t)c / (uint32_t)m.chunks_per_row;
+    r = rr;
+    k0 = (int64_t)((uint32_t)c - rr * (uint32_t)m.chunks_per_row) << 3;
+  } else {
+    r = c / m.chunks_per_row;
+    k0 = (c - r * m.chunks_per_row) << 3;
+  }
+}
 
 __global__ void __launch_bounds__(kThreads)
 absmax_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_row, int64_t K_pad,
                  int had_block, bool vec, float* amax_out, int32_t* dev_status) {
   const int64_t chunks_per_row = K_pad >> 3;
   const int64_t total = rows * chunks_per_row;
-  const int64_t total_warp = (total + 31) & ~int64_t(31);
+  const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
+  const bool dense = (K == K_pad) && (ld_row == K);
   const int lane = threadIdx.x & 31;
   uint32_t mx = 0u;
-  for (int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x; c < total_warp;
-       c += (int64_t)gridDim.x * kThreads) {
-    float x[8];
-    if (c < total) {
-      const int64_t r = c / chunks_per_row;
-      const int64_t k0 = (c - r * chunks_per_row) << 3;
-      load8_kc(src + r * ld_row, k0, K, vec, x);
-    } else {
+  for (int64_t base = (int64_t)blockIdx.x * (kThreads * kUnrollAbsmax); base < total;
+       base += (int64_t)gridDim.x * (kThreads * kUnrollAbsmax)) {
+    float x[kUnrollAbsmax][8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) x[i] = 0.0f;
+    for (int u = 0; u < kUnrollAbsmax; ++u) {
+      const int64_t c = base + u * kThreads + threadIdx.x;
+      if (c < total) {
+        if (dense) {   // rows are back to back and unpadded: chunk c starts at element 8c
+          load8_kc(src, c << 3, total << 3, vec, x[u]);
+        } else {
+          int64_t r, k0;
+          chunk_to_row_k(cmap, c, r, k0);
+          load8_kc(src + r * ld_row, k0, K, vec, x[u]);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[u][i] = 0.0f;
+      }
     }
-    fwht8_regs(x, had_block);
-    fwht8_lanes(x, had_block, lane);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) mx = max(mx, abs_bits(x[i]));
+    for (int u = 0; u < kUnrollAbsmax; ++u) {
+      fwht8_regs(x[u], had_block);
+      fwht8_lanes(x[u], had_block, lane);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mx = max(mx, abs_bits(x[u][i]));
+    }
   }
   block_absmax_commit(mx, amax_out, dev_status);
 }
@@ -231,52 +268,81 @@ quantize_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64
   }
   const int64_t chunks_per_row = K_pad >> 3;
   const int64_t total = rows * chunks_per_row;
-  const int64_t total_warp = (total + 31) & ~int64_t(31);
+  const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
+  const bool dense = (K == K_pad) && (ld_row == K);
   const int lane = threadIdx.x & 31;
-  for (int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x; c < total_warp;
-       c += (int64_t)gridDim.x * kThreads) {
-    float x[8];
-    const bool valid = c < total;
-    int64_t r = 0, k0 = 0;
-    if (valid) {
-      r = c / chunks_per_row;
-      k0 = (c - r * chunks_per_row) << 3;
-      load8_kc(src + r * ld_row, k0, K, vec, x);
-    } else {
+  for (int64_t base = (int64_t)blockIdx.x * (kThreads * kUnrollQuant); base < total;
+       base += (int64_t)gridDim.x * (kThreads * kUnrollQuant)) {
+    float x[kUnrollQuant][8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) x[i] = 0.0f;
-    }
-    fwht8_regs(x, had_block);
-    fwht8_lanes(x, had_block, lane);
-    int q[8];
-    quantize8(x, p, (uint64_t)c, q);  // linear index of the chunk's first element is 8*c
-    if (row_norms != nullptr) {
-      int ss = 0;
+    for (int u = 0; u < kUnrollQuant; ++u) {
+      const int64_t c = base + u * kThreads + threadIdx.x;
+      if (c < total) {
+        if (dense) {   // rows are back to back and unpadded: chunk c starts at element 8c
+          load8_kc(src, c << 3, total << 3, vec, x[u]);
+        } else {
+          int64_t r, k0;
+          chunk_to_row_k(cmap, c, r, k0);
+          load8_kc(src + r * ld_row, k0, K, vec, x[u]);
+        }
+      } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) ss += q[i] * q[i];
-      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
-      ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
-      if (valid && (lane & 3) == 0) row_norms[r * (K_pad >> 5) + (k0 >> 5)] = (uint16_t)ss;
+        for (int i = 0; i < 8; ++i) x[u][i] = 0.0f;
+      }
     }
-    if (valid) {
+#pragma unroll
+    for (int u = 0; u < kUnrollQuant; ++u) {
+      const int64_t c = base + u * kThreads + threadIdx.x;
+      const bool valid = c < total;
+      fwht8_regs(x[u], had_block);
+      fwht8_lanes(x[u], had_block, lane);
+      int q[8];
+      quantize8(x[u], p, (uint64_t)c, q);  // linear index of the chunk's first element is 8*c
+      // codes are dense [rows, K_pad]: chunk c is bytes [8c, 8c+8) and tile c/4 of the row-norm array
       uint2 out;
       out.x = pack4(q[0], q[1], q[2], q[3]);
       out.y = pack4(q[4], q[5], q[6], q[7]);
-      *reinterpret_cast<uint2*>(codes + r * K_pad + k0) = out;
+      if (row_norms != nullptr) {
+        int ss = __dp4a((int)out.x, (int)out.x, 0);
+        ss = __dp4a((int)out.y, (int)out.y, ss);
+        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+        if (valid && (lane & 3) == 0) row_norms[c >> 2] = (uint16_t)ss;
+      }
+      if (valid) *reinterpret_cast<uint2*>(codes + (c << 3)) = out;
     }
   }
 }
 
-// max over each block of 128 rows of the per-row tile norms
-__global__ void block_norms_kernel(const uint16_t* __restrict__ row_norms, int64_t rows, int64_t T,
-                                   int32_t* __restrict__ tile_norms) {
-  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+// max over each block of 128 rows of the per-row tile norms: a thread block covers 64 K tiles of one
+// row block, its 4 thread rows take 32 rows each, shared memory combines them
+__global__ void __launch_bounds__(256)
+block_norms_kernel(const uint16_t* __restrict__ row_norms, int64_t rows, int64_t T,
+                   int32_t* __restrict__ tile_norms) {
+  __shared__ int s_part[4][64];
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  const int64_t t = (int64_t)blockIdx.x * 64 + tx;
   const int64_t rb = blockIdx.y;
-  if (t >= T) return;
-  const int64_t r0 = rb * 128, r1 = min(rows, r0 + 128);
+  const int64_t r0 = rb * 128 + ty * 32;
   int mx = 0;
-  for (int64_t r = r0; r < r1; ++r) mx = max(mx, (int)row_norms[r * T + t]);
-  tile_norms[rb * T + t] = mx;
+  if (t < T) {
+    const uint16_t* p = row_norms + r0 * T + t;
+    if (r0 + 32 <= rows) {
+      // whole group in range: no per-row test, so the 32 independent loads can all be in flight
+      int v[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = (int)__ldg(p + i * T);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) mx = max(mx, v[i]);
+    } else {
+      for (int i = 0; i < 32 && r0 + i < rows; ++i) mx = max(mx, (int)__ldg(p + i * T));
+    }
+  }
+  s_part[ty][tx] = mx;
+  __syncthreads();
+  if (ty == 0 && t < T) {
+    tile_norms[rb * T + t] = max(max(s_part[0][tx], s_part[1][tx]), max(s_part[2][tx], s_part[3][tx]));
+  }
 }
 
 // ---- K-strided kernels ------------------------------------------------------------------------
@@ -295,16 +361,17 @@ __device__ __forceinline__ void load32_ks(const float* __restrict__ src, int64_t
   }
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 absmax_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_k, int64_t K_pad,
                  int had_block, float* amax_out, int32_t* dev_status) {
-  const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
-  const int64_t total = rows_pad * (K_pad >> 5);
+  // work item = (32-block of K, group of kThreads rows); the host guarantees that their number fits 31 bits
+  const uint32_t row_groups = (uint32_t)((rows + kThreads - 1) / kThreads);
+  const uint32_t items = row_groups * (uint32_t)(K_pad >> 5);
   uint32_t mx = 0u;
-  for (int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x; id < total;
-       id += (int64_t)gridDim.x * kThreads) {
-    const int64_t kb = id / rows_pad;
-    const int64_t r = id - kb * rows_pad;
+  for (uint32_t w = blockIdx.x; w < items; w += gridDim.x) {
+    const uint32_t kbu = w / row_groups;
+    const int64_t kb = kbu;
+    const int64_t r = (int64_t)(w - kbu * row_groups) * kThreads + threadIdx.x;
     if (r < rows) {
       float x[32];
       load32_ks(src, r, kb, K, ld_k, x);
@@ -316,7 +383,7 @@ absmax_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t
   block_absmax_commit(mx, amax_out, dev_status);
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_k, int64_t K_pad,
                    int had_block, int bits, float clip, int mode, uint64_t seed, uint32_t tag,
                    const float* __restrict__ amax_ptr, int8_t* __restrict__ codes, float* step_out,
@@ -330,14 +397,15 @@ quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64
   }
   // rows are padded to a multiple of the block size so that one thread block never straddles
   // two 32-blocks of K and always covers whole 128-row groups (needed for the tile norms)
-  const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
   const int64_t T = K_pad >> 5;
-  const int64_t total = rows_pad * T;
+  const uint32_t row_groups = (uint32_t)((rows + kThreads - 1) / kThreads);
+  const uint32_t items = row_groups * (uint32_t)T;   // the host guarantees that this fits 31 bits
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int64_t id0 = (int64_t)blockIdx.x * kThreads; id0 < total; id0 += (int64_t)gridDim.x * kThreads) {
-    const int64_t id = id0 + threadIdx.x;
-    const int64_t kb = id0 / rows_pad;          // uniform over the block
-    const int64_t r = id - kb * rows_pad;
+  for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
+    const uint32_t kbu = item / row_groups;     // uniform over the block
+    const int64_t kb = kbu;
+    const int64_t r_group0 = (int64_t)(item - kbu * row_groups) * kThreads;
+    const int64_t r = r_group0 + threadIdx.x;
     int ss = 0;
     if (r < rows) {
       float x[32];
@@ -352,10 +420,10 @@ quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64
 #pragma unroll
         for (int i = 0; i < 8; ++i) x8[i] = x[8 * j + i];
         quantize8(x8, p, g0 + j, q);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) ss += q[i] * q[i];
         w[2 * j] = pack4(q[0], q[1], q[2], q[3]);
         w[2 * j + 1] = pack4(q[4], q[5], q[6], q[7]);
+        ss = __dp4a((int)w[2 * j], (int)w[2 * j], ss);
+        ss = __dp4a((int)w[2 * j + 1], (int)w[2 * j + 1], ss);
       }
       uint4* dst = reinterpret_cast<uint4*>(codes + r * K_pad + (kb << 5));
       dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -367,7 +435,7 @@ quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64
       if (lane == 0) s_norm[warp] = ss;
       __syncthreads();
       if (threadIdx.x < kThreads / 128) {
-        const int64_t r_base = (id0 - kb * rows_pad) + threadIdx.x * 128;
+        const int64_t r_base = r_group0 + threadIdx.x * 128;
         if (r_base < rows) {
           int mx = 0;
 #pragma unroll
@@ -408,13 +476,13 @@ hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t l
   if (ld_k == 1) {
     const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
     const int64_t total = rows * (K_pad >> 3);
-    absmax_kc_kernel<<<grid_for(total, kThreads, 8), kThreads, 0, s>>>(src, rows, K, ld_row, K_pad, had_block,
-                                                                     vec, amax_out, dev_status);
+    absmax_kc_kernel<<<grid_for(total, kThreads * kUnrollAbsmax, 4), kThreads, 0, s>>>(
+        src, rows, K, ld_row, K_pad, had_block, vec, amax_out, dev_status);
   } else {
-    const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
-    const int64_t total = rows_pad * (K_pad >> 5);
-    absmax_ks_kernel<<<grid_for(total, kThreads, 4), kThreads, 0, s>>>(src, rows, K, ld_k, K_pad, had_block,
-                                                                     amax_out, dev_status);
+    const int64_t items = ((rows + kThreads - 1) / kThreads) * (K_pad >> 5);
+    if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
+    absmax_ks_kernel<<<grid_for(items, 1, 3), kThreads, 0, s>>>(src, rows, K, ld_k, K_pad, had_block, amax_out,
+                                                              dev_status);
   }
   return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
 }
@@ -430,17 +498,17 @@ hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t
     const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
     const int64_t total = rows * (K_pad >> 3);
     uint16_t* rn = tile_norms ? row_norms_scratch : nullptr;
-    quantize_kc_kernel<<<grid_for(total, kThreads, 8), kThreads, 0, s>>>(
+    quantize_kc_kernel<<<grid_for(total, kThreads * kUnrollQuant, 4), kThreads, 0, s>>>(
         src, rows, K, ld_row, K_pad, had_block, vec, bits, clip, mode, seed, tag, amax, codes, step_out, rn,
         dev_status);
     if (tile_norms) {
-      dim3 grid((unsigned)((T + 127) / 128), (unsigned)((rows + 127) / 128));
-      block_norms_kernel<<<grid, 128, 0, s>>>(rn, rows, T, tile_norms);
+      dim3 grid((unsigned)((T + 63) / 64), (unsigned)((rows + 127) / 128));
+      block_norms_kernel<<<grid, 256, 0, s>>>(rn, rows, T, tile_norms);
     }
   } else {
-    const int64_t rows_pad = (rows + kThreads - 1) / kThreads * kThreads;
-    const int64_t total = rows_pad * T;
-    quantize_ks_kernel<<<grid_for(total, kThreads, 4), kThreads, 0, s>>>(
+    const int64_t items = ((rows + kThreads - 1) / kThreads) * T;
+    if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
+    quantize_ks_kernel<<<grid_for(items, 1, 3), kThreads, 0, s>>>(
         src, rows, K, ld_k, K_pad, had_block, bits, clip, mode, seed, tag, amax, codes, step_out, tile_norms,
         dev_status);
   }
