@@ -28,6 +28,9 @@ sys.path.insert(0, ROOT)
 METRIC = "hdqt_gemm_int_tops"
 UNIT = "TOPS"
 SEED = 1234
+# dram__bytes_read.sum + dram__bytes_write.sum of one gemm_i8_tiled_kernel launch at M=N=K=8192 (merged path),
+# from the ncu capture summarised in profiles/gemm_i8_tiled_kernel_sweep.md
+GEMM_DRAM_BYTES_8192 = 344.4e6 + 238.0e6
 
 
 def parse_args():
@@ -308,7 +311,10 @@ def run_hdqt(args):
             "data": "synthetic", "config": workload_config(size, merge),
             "roofline": {"bound": "tensor", "kernel": "gemm_i8_tiled_kernel", "achieved": gemm_tops,
                          "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak, "peak_source": peak_src,
-                         "traffic": None, "ms_per_launch": gemm_ms},
+                         "traffic": GEMM_DRAM_BYTES_8192 if (size == 8192 and merge) else None,
+                         "traffic_unit": "bytes per launch (ncu dram read+write, profiles/gemm_i8_tiled_kernel_sweep.md)",
+                         "algorithmic_bytes": float(M * K + N * K + 4 * M * N),
+                         "ms_per_launch": gemm_ms},
             "quantize": {"ms_per_step": quant_ms, "algorithmic_gb_per_step": quant_bytes / 1e9,
                          "gbs": quant_bytes / (quant_ms * 1e-3) / 1e9, "hbm_peak_gbs": hbm,
                          "frac": quant_bytes / (quant_ms * 1e-3) / 1e9 / hbm,
