@@ -172,6 +172,22 @@ def run_reference(args):
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of per-rank timings over all ranks (every rank gets the result)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_tops(world, steps, ops_per_step, elapsed_ms):
+    """Aggregate throughput of `world` replicas that each ran `steps` steps in `elapsed_ms` (max over ranks)."""
+    return world * steps * ops_per_step / (elapsed_ms * 1e-3) / 1e12
+
+
 def run_hdqt(args):
     import torch
     import torch.distributed as dist
@@ -276,19 +292,13 @@ def run_hdqt(args):
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = t.item()
-        e2e = {"value": world * e2e_steps * 2.0 * M * N * K / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+        e2e_ms = max_over_ranks([e2e_ms], dev, world)[0]
+        e2e = {"value": whole_job_tops(world, e2e_steps, 2.0 * M * N * K, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": hA.numel() * 4 + hB.numel() * 4, "d2h_bytes_per_step": hOut.numel() * 4,
                "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps}
         hdqt.check_device_status(status, "e2e")
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms, quant_ms, gemm_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, quant_ms, gemm_ms = t.tolist()
+    elapsed_ms, quant_ms, gemm_ms = max_over_ranks([elapsed_ms, quant_ms, gemm_ms], dev, world)
 
     if rank == 0:
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -305,7 +315,7 @@ def run_hdqt(args):
         gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
         quant_bytes = 9.0 * (M * K + N * K)      # 4 B calibration read + 4 B read + 1 B code written, per element
         line = {
-            "metric": METRIC, "value": world * args.steps * ops / (elapsed_ms * 1e-3) / 1e12, "unit": UNIT,
+            "metric": METRIC, "value": whole_job_tops(world, args.steps, ops, elapsed_ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32",
             "data": "synthetic", "config": workload_config(size, merge),
