@@ -40,18 +40,21 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="hdqt", choices=["hdqt", "reference"])
     ap.add_argument("--size", type=int, default=8192, help="M = N = K of the sweep shape")
+    ap.add_argument("--layout", default="dgrad", choices=["dgrad", "wgrad"],
+                    help="dgrad: both operands K-contiguous, A stochastic / B nearest; "
+                         "wgrad: both operands K-strided (transposed reads), both stochastic")
     ap.add_argument("--no-merge", action="store_true", help="disable merging of provably clamp-free tiles")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     return ap.parse_args()
 
 
-def workload_config(size: int, merge: bool):
+def workload_config(size: int, merge: bool, layout: str = "dgrad"):
     return {
-        "workload": f"roofline-sweep dgrad-layout HDQT GEMM M=N=K={size} (Student-t(3), 0.1% outliers x50)",
+        "workload": f"roofline-sweep {layout}-layout HDQT GEMM M=N=K={size} (Student-t(3), 0.1% outliers x50)",
         "M": size, "N": size, "K": size,
         "in_bits": 4, "acc_bits": 8, "acc_tile": 32, "had_block": 32, "acc_shift": 0,
-        "rounding": "A stochastic (Philox4x32-10), B nearest",
+        "rounding": "A stochastic (Philox4x32-10), B nearest" if layout == "dgrad" else "A and B stochastic (Philox4x32-10)",
         "clamp_free_tile_merging": bool(merge),
         "l2": "inputs_exceed_l2" if size * size * 4 > 126 * 2 ** 20 else "inputs_within_l2_not_flushed",
         "parallelism": "replicas",
@@ -110,7 +113,7 @@ class ClockSampler:
 # CPU oracle arm (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
 
-def oracle_sample_run(size: int, rows_a: int, rows_b: int, seed: int):
+def oracle_sample_run(size: int, rows_a: int, rows_b: int, seed: int, layout: str = "dgrad"):
     """One pass of the oracle over a slice of the workload: rows_a rows of A, rows_b rows of B, full K.
     Returns (seconds, equivalent integer ops)."""
     from oracle import hdqt_oracle as O
@@ -118,7 +121,10 @@ def oracle_sample_run(size: int, rows_a: int, rows_b: int, seed: int):
     A = inputs.heavy_tailed(rows_a, size, seed)
     B = inputs.heavy_tailed(rows_b, size, seed + 1)
     t0 = time.perf_counter()
-    O.gemm_dgrad(A, B, O.dgrad_desc(seed=seed))
+    if layout == "wgrad":
+        O.gemm_wgrad(np.ascontiguousarray(A.T), np.ascontiguousarray(B.T), O.wgrad_desc(seed=seed))
+    else:
+        O.gemm_dgrad(A, B, O.dgrad_desc(seed=seed))
     dt = time.perf_counter() - t0
     return dt, 2.0 * rows_a * rows_b * size
 
@@ -132,9 +138,9 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def cpu_baseline(size: int):
+def cpu_baseline(size: int, layout: str = "dgrad"):
     rows_a, rows_b = min(size, 1024), min(size, 2048)
-    dt, ops = oracle_sample_run(size, rows_a, rows_b, SEED)
+    dt, ops = oracle_sample_run(size, rows_a, rows_b, SEED, layout)
     return {"value": ops / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
             "seconds": dt,
             "sample": f"{rows_a} rows of A x {rows_b} rows of B, full K={size} (whole path: FWHT, quantize, "
@@ -148,10 +154,10 @@ def run_reference(args):
     size = args.size
     rows_a, rows_b = min(size, 256), min(size, 512)
     for _ in range(min(args.warmup, 1)):
-        oracle_sample_run(size, rows_a, rows_b, SEED)
+        oracle_sample_run(size, rows_a, rows_b, SEED, args.layout)
     total_t, total_ops = 0.0, 0.0
     for i in range(args.steps):
-        dt, ops = oracle_sample_run(size, rows_a, rows_b, SEED + i)
+        dt, ops = oracle_sample_run(size, rows_a, rows_b, SEED + i, args.layout)
         total_t += dt
         total_ops += ops
     value = total_ops / total_t / 1e12
@@ -160,7 +166,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_t / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32", "data": "synthetic",
-        "config": workload_config(size, not args.no_merge),
+        "config": workload_config(size, not args.no_merge, args.layout),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -205,11 +211,16 @@ def run_hdqt(args):
     M = N = K = size
     merge = not args.no_merge
     flags = 0 if merge else hdqt.FLAG_NO_MERGE
-    desc = hdqt.default_desc("dgrad", seed=SEED, flags=flags)
+    wgrad = args.layout == "wgrad"
+    desc = hdqt.default_desc("wgrad" if wgrad else "dgrad", seed=SEED, flags=flags)
 
     # every rank works on its own operands (independent problems: no data-path collective)
     A = inputs.heavy_tailed_torch(M, K, SEED + 10 * rank, dev)
     B = inputs.heavy_tailed_torch(N, K, SEED + 10 * rank + 1, dev)
+    if wgrad:
+        # dW = X^T G: the operands are stored [K, M] and [K, N] (contraction index strided)
+        Xs, Gs = A.t().contiguous(), B.t().contiguous()
+        A, B = Xs.t(), Gs.t()          # logical [M, K] / [N, K] views with stride (1, M) / (1, N)
     out = torch.empty((M, N), dtype=torch.float32, device=dev)
     status = hdqt.new_status(dev)
     Kp = hdqt.padded_k(K)
@@ -268,19 +279,21 @@ def run_hdqt(args):
     # end to end through the public call with host buffers: H2D of both operands, D2H of the result
     e2e = None
     if not args.skip_e2e:
-        hA = torch.empty((M, K), dtype=torch.float32).pin_memory()
-        hB = torch.empty((N, K), dtype=torch.float32).pin_memory()
-        hA.copy_(A)
-        hB.copy_(B)
+        srcA, srcB = (Xs, Gs) if wgrad else (A, B)
+        hA = torch.empty(tuple(srcA.shape), dtype=torch.float32).pin_memory()
+        hB = torch.empty(tuple(srcB.shape), dtype=torch.float32).pin_memory()
+        hA.copy_(srcA)
+        hB.copy_(srcB)
         hOut = torch.empty((M, N), dtype=torch.float32).pin_memory()
-        dA, dB = torch.empty_like(A), torch.empty_like(B)
+        dA, dB = torch.empty_like(srcA), torch.empty_like(srcB)
         ws = hdqt.Workspace(desc, M, N, K, dev)
         e2e_steps = max(3, min(args.steps, 5))
+        public_call = hdqt.gemm_wgrad if wgrad else hdqt.gemm_dgrad
 
         def e2e_step():
             dA.copy_(hA, non_blocking=True)
             dB.copy_(hB, non_blocking=True)
-            hdqt.gemm_dgrad(dA, dB, desc=desc, workspace=ws, dev_status=status, out=out)
+            public_call(dA, dB, desc=desc, workspace=ws, dev_status=status, out=out)
             hOut.copy_(out, non_blocking=True)
 
         e2e_step()
@@ -318,10 +331,10 @@ def run_hdqt(args):
             "metric": METRIC, "value": whole_job_tops(world, args.steps, ops, elapsed_ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32",
-            "data": "synthetic", "config": workload_config(size, merge),
+            "data": "synthetic", "config": workload_config(size, merge, args.layout),
             "roofline": {"bound": "tensor", "kernel": "gemm_i8_tiled_kernel", "achieved": gemm_tops,
                          "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak, "peak_source": peak_src,
-                         "traffic": GEMM_DRAM_BYTES_8192 if (size == 8192 and merge) else None,
+                         "traffic": GEMM_DRAM_BYTES_8192 if (size == 8192 and merge and not wgrad) else None,
                          "traffic_unit": "bytes per launch (ncu dram read+write, profiles/gemm_i8_tiled_kernel_sweep.md)",
                          "algorithmic_bytes": float(M * K + N * K + 4 * M * N),
                          "ms_per_launch": gemm_ms},
@@ -329,12 +342,12 @@ def run_hdqt(args):
                          "gbs": quant_bytes / (quant_ms * 1e-3) / 1e9, "hbm_peak_gbs": hbm,
                          "frac": quant_bytes / (quant_ms * 1e-3) / 1e9 / hbm,
                          "note": "both operands: calibration pass (4 B/elt) + FWHT/quantize pass (5 B/elt)"},
-            "clocks": clocks, "gpu_launches": args.steps * (5 + (2 if merge else 0)),
+            "clocks": clocks, "gpu_launches": args.steps * (5 + (2 if (merge and not wgrad) else 0)),
         }
         if e2e is not None:
             line["e2e"] = e2e
         if not args.skip_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(size)
+            line["cpu_baseline"] = cpu_baseline(size, args.layout)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

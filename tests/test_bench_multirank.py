@@ -47,7 +47,7 @@ def test_reference_arm_prints_on_rank0_only(capsys, monkeypatch):
     import bench
 
     class A:
-        size, steps, warmup, gpus, no_merge = 256, 1, 0, 2, False
+        size, steps, warmup, gpus, no_merge, layout = 256, 1, 0, 2, False, "dgrad"
 
     monkeypatch.setenv("RANK", "1")
     bench.run_reference(A)

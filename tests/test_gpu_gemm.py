@@ -208,9 +208,11 @@ def test_runs_are_bitwise_reproducible(hdqt):
     assert not torch.equal(a, c)
 
 
-def test_sampled_parity_at_sweep_size(hdqt):
-    """4096^3 dgrad-layout GEMM on heavy-tailed operands: codes in full, integer sums on sampled rows/columns."""
-    M = N = K = 4096
+@pytest.mark.parametrize("size", [4096, 8192])
+def test_sampled_parity_at_sweep_size(hdqt, size):
+    """Sweep-size dgrad-layout GEMM on heavy-tailed operands (8192 = the shape and launch configuration the
+    benchmark times): codes in full, outputs on sampled rows and columns."""
+    M = N = K = size
     A = inputs.heavy_tailed_torch(M, K, seed=100, device="cuda")
     B = inputs.heavy_tailed_torch(N, K, seed=101, device="cuda")
     desc = hdqt.default_desc("dgrad", seed=9)
@@ -312,3 +314,44 @@ def test_wide_accumulators_merge_without_norms(hdqt):
     for acc_bits in (13, 16, 32):
         _, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), one, one, acc_bits, 32, 0, 32, want_S=True)
         assert np.array_equal(S.cpu().numpy().astype(np.int64), plain)
+
+
+def test_sampled_parity_wgrad_layout_at_sweep_size(hdqt):
+    """4096^3 wgrad layout (both operands K-strided, both stochastic): codes in full, outputs sampled."""
+    M = N = K = 4096
+    X = inputs.heavy_tailed_torch(K, M, seed=200, device="cuda")     # stored [Nb, D]: contraction index first
+    G = inputs.heavy_tailed_torch(K, N, seed=201, device="cuda")
+    desc = hdqt.default_desc("wgrad", seed=5)
+    status = hdqt.new_status("cuda")
+    out, ws = hdqt.gemm_wgrad(X, G, desc=desc, dev_status=status)
+    hdqt.check_device_status(status)
+    want_a, sa, _ = O.quantize_hadamard(X.cpu().numpy().T, 32, 4, 1.0, 1, seed=5, tag=desc.tag_a)
+    want_b, sb, _ = O.quantize_hadamard(G.cpu().numpy().T, 32, 4, 1.0, 1, seed=5, tag=desc.tag_b)
+    assert np.array_equal(ws.codes_a().cpu().numpy(), want_a)
+    assert np.array_equal(ws.codes_b().cpu().numpy(), want_b)
+    rng = np.random.default_rng(1)
+    rows = np.sort(rng.choice(M, 48, replace=False))
+    cols = np.sort(rng.choice(N, 48, replace=False))
+    got = out.cpu().numpy()
+    want_rows, _, _ = O.gemm_i8_tiled(want_a[rows], want_b, sa, sb)
+    want_cols, _, _ = O.gemm_i8_tiled(want_a, want_b[cols], sa, sb)
+    assert np.array_equal(got[rows], want_rows) and np.array_equal(got[:, cols], want_cols)
+
+
+def test_tall_skinny_conv_like_shapes(hdqt):
+    """im2col-like layer: 32768 x 576 activations, 64 output channels (many row blocks, one column block)."""
+    Nb, D, C = 32768, 576, 64
+    X = np.maximum(inputs.activations(Nb, D, seed=31), 0)
+    W = inputs.weights(D, C, seed=32)
+    G = inputs.gradients(Nb, C, seed=33)
+    status = hdqt.new_status("cuda")
+    Xd, Wd, Gd = _dev(X), _dev(W), _dev(G)
+    for kind, fn, args, want in (
+            ("fwd", hdqt.gemm_fwd, (Xd, Wd), O.gemm_fwd(X, W, O.fwd_desc(tag_a=0, tag_b=1, seed=2))),
+            ("dgrad", hdqt.gemm_dgrad, (Gd, Wd), O.gemm_dgrad(G, W, O.dgrad_desc(tag_a=2, tag_b=3, seed=2))),
+            ("wgrad", hdqt.gemm_wgrad, (Xd, Gd), O.gemm_wgrad(X, G, O.wgrad_desc(tag_a=4, tag_b=5, seed=2)))):
+        out, ws = fn(*args, desc=hdqt.default_desc(kind, seed=2), dev_status=status)
+        hdqt.check_device_status(status, kind)
+        assert np.array_equal(ws.codes_a().cpu().numpy(), want["Aq"]), kind
+        assert np.array_equal(ws.codes_b().cpu().numpy(), want["Bq"]), kind
+        _assert_close(out.cpu().numpy(), want["out"])
