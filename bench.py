@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--layout", default="dgrad", choices=["dgrad", "wgrad"],
                     help="dgrad: both operands K-contiguous, A stochastic / B nearest; "
                          "wgrad: both operands K-strided (transposed reads), both stochastic")
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "mlp"],
+                    help="sweep: the GEMM roofline shape (default, the headline line); mlp: training steps/s of the "
+                         "synthetic 1152-512-256-12 MLP, batch 256 (a secondary report)")
     ap.add_argument("--no-merge", action="store_true", help="disable merging of provably clamp-free tiles")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -353,10 +356,44 @@ def run_hdqt(args):
         dist.destroy_process_group()
 
 
+def run_mlp(args):
+    """Training steps/s of the synthetic MLP step (every matmul through the library), with the fp32 torch
+    step of the same model as context. Secondary report: one JSON line of its own."""
+    import torch
+    from paper_2310_03675_b200 import nn as hnn
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    x, labels = hnn.sensor_window_batch(256, 1152, 12, seed=SEED, device=dev)
+    out = {}
+    for name, quantized in (("hdqt", True), ("fp32_torch", False)):
+        torch.manual_seed(0)
+        model = hnn.Mlp(quantized=quantized).to(dev)
+        opt = torch.optim.SGD(model.parameters(), lr=0.01, momentum=0.9)
+        for i in range(max(args.warmup, 3)):
+            hnn.train_step(model, opt, x, labels, i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            loss = hnn.train_step(model, opt, x, labels, 1000 + i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        out[name] = {"steps_per_s": 1e3 / ms, "ms_per_step": ms, "final_loss": float(loss.item())}
+    print(json.dumps({"metric": "hdqt_mlp_train_steps_per_s", "value": out["hdqt"]["steps_per_s"], "unit": "steps/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+                      "ms_per_step": out["hdqt"]["ms_per_step"], "higher_is_better": True, "data": "synthetic",
+                      "config": {"workload": "MLP 1152-512-256-12, batch 256, SGD momentum 0.9, 4-bit inputs, "
+                                             "8-bit accumulators, Hadamard block 32"},
+                      "fp32_torch": out["fp32_torch"], "hdqt": out["hdqt"]}))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "mlp":
+        run_mlp(args)
     else:
         run_hdqt(args)
 

@@ -179,24 +179,41 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
   int32_t* normsB = merge ? reinterpret_cast<int32_t*>(ws + L.norms_b) : nullptr;
   const size_t scratch_bytes = L.total - L.gemm_ws;
 
-  st = hdqt_quantize_hadamard(gA.src, gA.rows, K, gA.ld_row, gA.ld_k, d->had_block, d->in_bits, clipA, roundA,
-                              d->seed, tagA, amaxA, reinterpret_cast<int8_t*>(ws + L.codes_a),
-                              reinterpret_cast<float*>(ws + L.step_a), normsA, ws + L.gemm_ws, scratch_bytes,
-                              dev_status, stream);
-  if (st != HDQT_OK) return st;
-  // keep the measured maxima where the layout says (for harnesses that read them back)
+  // argument rules of hdqt_quantize_hadamard, checked once for both operands
+  if ((st = check_quant_args(gA.src, gA.rows, K, gA.ld_row, gA.ld_k, d->had_block)) != HDQT_OK) return st;
+  if ((st = check_quant_args(gB.src, gB.rows, K, gB.ld_row, gB.ld_k, d->had_block)) != HDQT_OK) return st;
+  if (d->in_bits < 2 || d->in_bits > 8) return HDQT_ERR_INVALID_ARG;
+  if (!(clipA >= 1.0f / 64.0f && clipA <= 1.0f) || !(clipB >= 1.0f / 64.0f && clipB <= 1.0f))
+    return HDQT_ERR_INVALID_ARG;
+  if ((roundA != HDQT_ROUND_NEAREST && roundA != HDQT_ROUND_STOCHASTIC) ||
+      (roundB != HDQT_ROUND_NEAREST && roundB != HDQT_ROUND_STOCHASTIC))
+    return HDQT_ERR_INVALID_ARG;
+
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  if (!amaxA && cudaMemcpyAsync(ws + L.amax_a, ws + L.gemm_ws, sizeof(float), cudaMemcpyDeviceToDevice, s) !=
-                    cudaSuccess)
-    return HDQT_ERR_CUDA;
-  st = hdqt_quantize_hadamard(gB.src, gB.rows, K, gB.ld_row, gB.ld_k, d->had_block, d->in_bits, clipB, roundB,
-                              d->seed, tagB, amaxB, reinterpret_cast<int8_t*>(ws + L.codes_b),
-                              reinterpret_cast<float*>(ws + L.step_b), normsB, ws + L.gemm_ws, scratch_bytes,
-                              dev_status, stream);
+  // measured maxima live where the layout says (harnesses read them back); both are cleared by one memset
+  float* amax_slot_a = reinterpret_cast<float*>(ws + L.amax_a);
+  float* amax_slot_b = reinterpret_cast<float*>(ws + L.amax_b);
+  if (!amaxA || !amaxB) {
+    if (cudaMemsetAsync(ws + L.amax_a, 0, (L.amax_b - L.amax_a) + sizeof(float), s) != cudaSuccess) return HDQT_ERR_CUDA;
+  }
+  uint16_t* row_norms = reinterpret_cast<uint16_t*>(ws + L.gemm_ws);
+  if (scratch_bytes < hdqt_quantize_workspace_bytes(M > N ? M : N, K, d->had_block)) return HDQT_ERR_WORKSPACE;
+  if (!amaxA) {
+    st = launch_absmax(gA.src, gA.rows, K, gA.ld_row, gA.ld_k, d->had_block, amax_slot_a, dev_status, s, false);
+    if (st != HDQT_OK) return st;
+  }
+  if (!amaxB) {
+    st = launch_absmax(gB.src, gB.rows, K, gB.ld_row, gB.ld_k, d->had_block, amax_slot_b, dev_status, s, false);
+    if (st != HDQT_OK) return st;
+  }
+  st = launch_quantize(gA.src, gA.rows, K, gA.ld_row, gA.ld_k, d->had_block, d->in_bits, clipA, roundA, d->seed, tagA,
+                       amaxA ? amaxA : amax_slot_a, reinterpret_cast<int8_t*>(ws + L.codes_a),
+                       reinterpret_cast<float*>(ws + L.step_a), normsA, row_norms, dev_status, s);
   if (st != HDQT_OK) return st;
-  if (!amaxB && cudaMemcpyAsync(ws + L.amax_b, ws + L.gemm_ws, sizeof(float), cudaMemcpyDeviceToDevice, s) !=
-                    cudaSuccess)
-    return HDQT_ERR_CUDA;
+  st = launch_quantize(gB.src, gB.rows, K, gB.ld_row, gB.ld_k, d->had_block, d->in_bits, clipB, roundB, d->seed, tagB,
+                       amaxB ? amaxB : amax_slot_b, reinterpret_cast<int8_t*>(ws + L.codes_b),
+                       reinterpret_cast<float*>(ws + L.step_b), normsB, row_norms, dev_status, s);
+  if (st != HDQT_OK) return st;
   return hdqt_gemm_i8_tiled(reinterpret_cast<int8_t*>(ws + L.codes_a), reinterpret_cast<int8_t*>(ws + L.codes_b),
                             reinterpret_cast<float*>(ws + L.step_a), reinterpret_cast<float*>(ws + L.step_b), M, N,
                             L.k_pad, d->in_bits, d->acc_bits, d->acc_tile, d->acc_shift, d->had_block, out, ld_out, nullptr,

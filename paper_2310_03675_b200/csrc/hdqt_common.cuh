@@ -68,8 +68,10 @@ inline hdqt_status_t cuda_failure(cudaError_t e, const char* what) {
 }
 
 // ---- internal launchers (defined in the .cu files) ----
+// zero_first = false: the caller has already cleared *amax_out on the stream
 hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
-                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s);
+                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s,
+                            bool zero_first = true);
 
 hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
                               int32_t had_block, int32_t bits, float clip, int32_t mode, uint64_t seed,

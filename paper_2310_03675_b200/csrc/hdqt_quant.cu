@@ -470,9 +470,10 @@ static int grid_for(int64_t work_items, int per_block, int blocks_per_sm) {
 }
 
 hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
-                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s) {
+                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s,
+                            bool zero_first) {
   const int64_t K_pad = hdqt_padded_k(K, had_block);
-  if (cudaMemsetAsync(amax_out, 0, sizeof(float), s) != cudaSuccess) return HDQT_ERR_CUDA;
+  if (zero_first && cudaMemsetAsync(amax_out, 0, sizeof(float), s) != cudaSuccess) return HDQT_ERR_CUDA;
   if (ld_k == 1) {
     const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
     const int64_t total = rows * (K_pad >> 3);
