@@ -46,17 +46,19 @@ def parse_args():
     ap.add_argument("--workload", default="sweep", choices=["sweep", "mlp"],
                     help="sweep: the GEMM roofline shape (default, the headline line); mlp: training steps/s of the "
                          "synthetic 1152-512-256-12 MLP, batch 256 (a secondary report)")
+    ap.add_argument("--acc-tile", type=int, default=32, help="accumulator tile length s along K (0 = whole K)")
+    ap.add_argument("--acc-bits", type=int, default=8, help="accumulator bit width b_a")
     ap.add_argument("--no-merge", action="store_true", help="disable merging of provably clamp-free tiles")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     return ap.parse_args()
 
 
-def workload_config(size: int, merge: bool, layout: str = "dgrad"):
+def workload_config(size: int, merge: bool, layout: str = "dgrad", acc_tile: int = 32, acc_bits: int = 8):
     return {
         "workload": f"roofline-sweep {layout}-layout HDQT GEMM M=N=K={size} (Student-t(3), 0.1% outliers x50)",
         "M": size, "N": size, "K": size,
-        "in_bits": 4, "acc_bits": 8, "acc_tile": 32, "had_block": 32, "acc_shift": 0,
+        "in_bits": 4, "acc_bits": acc_bits, "acc_tile": acc_tile, "had_block": 32, "acc_shift": 0,
         "rounding": "A stochastic (Philox4x32-10), B nearest" if layout == "dgrad" else "A and B stochastic (Philox4x32-10)",
         "clamp_free_tile_merging": bool(merge),
         "l2": "inputs_exceed_l2" if size * size * 4 > 126 * 2 ** 20 else "inputs_within_l2_not_flushed",
@@ -169,7 +171,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_t / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32", "data": "synthetic",
-        "config": workload_config(size, not args.no_merge, args.layout),
+        "config": workload_config(size, not args.no_merge, args.layout, args.acc_tile, args.acc_bits),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -215,7 +217,8 @@ def run_hdqt(args):
     merge = not args.no_merge
     flags = 0 if merge else hdqt.FLAG_NO_MERGE
     wgrad = args.layout == "wgrad"
-    desc = hdqt.default_desc("wgrad" if wgrad else "dgrad", seed=SEED, flags=flags)
+    desc = hdqt.default_desc("wgrad" if wgrad else "dgrad", seed=SEED, flags=flags, acc_tile=args.acc_tile,
+                             acc_bits=args.acc_bits)
 
     # every rank works on its own operands (independent problems: no data-path collective)
     A = inputs.heavy_tailed_torch(M, K, SEED + 10 * rank, dev)
@@ -316,6 +319,20 @@ def run_hdqt(args):
 
     elapsed_ms, quant_ms, gemm_ms = max_over_ranks([elapsed_ms, quant_ms, gemm_ms], dev, world)
 
+    certified = None
+    if merge and bufA[2] is not None and desc.acc_tile == 32 and rank == 0:
+        # fraction of (128x256 output block, K tile) pairs whose Cauchy-Schwarz bound proves "no clamp"
+        na = bufA[2].to(torch.int64)                                    # [M/128, T]
+        nb = bufB[2].to(torch.int64)
+        if nb.shape[0] % 2:
+            nb = torch.cat([nb, torch.zeros_like(nb[:1])])
+        nb = nb.view(-1, 2, nb.shape[1]).amax(1)                        # [N/256, T]
+        hi = (1 << (desc.acc_bits - 1)) - 1
+        cert = 0
+        for i in range(na.shape[0]):
+            cert += int(((na[i][None, :] * nb) <= hi * hi).sum().item())
+        certified = cert / float(na.shape[0] * nb.shape[0] * nb.shape[1])
+
     if rank == 0:
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
         if os.path.exists(peaks_path):
@@ -334,13 +351,13 @@ def run_hdqt(args):
             "metric": METRIC, "value": whole_job_tops(world, args.steps, ops, elapsed_ms), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32",
-            "data": "synthetic", "config": workload_config(size, merge, args.layout),
+            "data": "synthetic", "config": workload_config(size, merge, args.layout, args.acc_tile, args.acc_bits),
             "roofline": {"bound": "tensor", "kernel": "gemm_i8_tiled_kernel", "achieved": gemm_tops,
                          "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak, "peak_source": peak_src,
                          "traffic": GEMM_DRAM_BYTES_8192 if (size == 8192 and merge and not wgrad) else None,
                          "traffic_unit": "bytes per launch (ncu dram read+write, profiles/gemm_i8_tiled_kernel_sweep.md)",
                          "algorithmic_bytes": float(M * K + N * K + 4 * M * N),
-                         "ms_per_launch": gemm_ms},
+                         "ms_per_launch": gemm_ms, "certified_clamp_free_tile_fraction": certified},
             "quantize": {"ms_per_step": quant_ms, "algorithmic_gb_per_step": quant_bytes / 1e9,
                          "gbs": quant_bytes / (quant_ms * 1e-3) / 1e9, "hbm_peak_gbs": hbm,
                          "frac": quant_bytes / (quant_ms * 1e-3) / 1e9 / hbm,

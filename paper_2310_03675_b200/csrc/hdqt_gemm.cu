@@ -466,36 +466,85 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           merged_started = 1u;
           acc += 4;    // only meaningful (and only used) when tiles_per_acc == 1
         } else {
-          const int kt1 = min(tiles32, kt0 + 4);
-          for (int kt = kt0; kt < kt1; ++kt) {
-            if (j == 0) {
-              if (p.merge == 2) {
-                cert = true;
-              } else if (merging) {
-                cert = (cert_mask[acc >> 5] >> (acc & 31)) & 1u;
+          if (tpa < 4) {
+            // short accumulator tiles: one MMA per pass keeps this thread's path between a released
+            // accumulator and the next MMA as short as possible (it is on the critical chain of every tile)
+            const int kt1 = min(tiles32, kt0 + 4);
+            for (int kt = kt0; kt < kt1; ++kt) {
+              if (j == 0) {
+                if (p.merge == 2) {
+                  cert = true;
+                } else if (merging) {
+                  cert = (cert_mask[acc >> 5] >> (acc & 31)) & 1u;
+                }
+                if (cert) {
+                  d_tmem = tmem_base;                      // merged tiles accumulate in buffer 0
+                } else {
+                  // clamp tiles: buffer 1 when merging, else alternate 0 / 1
+                  const int buf = merging ? 1 : (clamp_idx & 1);
+                  const uint32_t use = merging ? (uint32_t)clamp_idx : (uint32_t)(clamp_idx >> 1);
+                  if (!mbar_wait(bar_tempty + 8 * buf, (use & 1) ^ 1, abort_flag)) { ok = false; break; }
+                  tc_fence_after();
+                  d_tmem = tmem_base + buf * BN;
+                  tfull_bar = bar_tfull + 8 * buf;
+                }
               }
-              if (cert) {
-                d_tmem = tmem_base;                      // merged tiles accumulate in buffer 0
-              } else {
-                // clamp tiles: buffer 1 when merging, else alternate 0 / 1
-                const int buf = merging ? 1 : (clamp_idx & 1);
-                const uint32_t use = merging ? (uint32_t)clamp_idx : (uint32_t)(clamp_idx >> 1);
-                if (!mbar_wait(bar_tempty + 8 * buf, (use & 1) ^ 1, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                d_tmem = tmem_base + buf * BN;
-                tfull_bar = bar_tfull + 8 * buf;
+              const uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
+              tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, cert ? merged_started : (uint32_t)(j != 0));
+              if (cert) merged_started = 1u;
+              if (++j == tpa || kt == tiles32 - 1) {
+                if (!cert) {
+                  tc_commit(tfull_bar);
+                  ++clamp_idx;
+                }
+                j = 0;
+                ++acc;
               }
             }
-            const uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
-            tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, cert ? merged_started : (uint32_t)(j != 0));
-            if (cert) merged_started = 1u;
-            if (++j == tpa || kt == tiles32 - 1) {
-              if (!cert) {
-                tc_commit(tfull_bar);
-                ++clamp_idx;
+          } else {
+            // long accumulator tiles: the K tiles of this stage that belong to the current accumulator
+            // tile go out back to back
+            const int kt1 = min(tiles32, kt0 + 4);
+            int kt = kt0;
+            while (kt < kt1) {
+              if (j == 0) {
+                if (p.merge == 2) {
+                  cert = true;
+                } else if (merging) {
+                  cert = (cert_mask[acc >> 5] >> (acc & 31)) & 1u;
+                }
+                if (cert) {
+                  d_tmem = tmem_base;                      // merged tiles accumulate in buffer 0
+                } else {
+                  // clamp tiles: buffer 1 when merging, else alternate 0 / 1
+                  const int buf = merging ? 1 : (clamp_idx & 1);
+                  const uint32_t use = merging ? (uint32_t)clamp_idx : (uint32_t)(clamp_idx >> 1);
+                  if (!mbar_wait(bar_tempty + 8 * buf, (use & 1) ^ 1, abort_flag)) { ok = false; break; }
+                  tc_fence_after();
+                  d_tmem = tmem_base + buf * BN;
+                  tfull_bar = bar_tfull + 8 * buf;
+                }
               }
-              j = 0;
-              ++acc;
+              // the K tiles of this stage that belong to the current accumulator tile go out back to back
+              uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
+              uint32_t accumulate = cert ? merged_started : (uint32_t)(j != 0);
+              const int run = min(kt1 - kt, tpa - j);
+              for (int i = 0; i < run; ++i) {
+                tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, accumulate);
+                sub2 += 2;
+                accumulate = 1u;
+              }
+              if (cert) merged_started = 1u;
+              j += run;
+              kt += run;
+              if (j == tpa || kt == tiles32) {
+                if (!cert) {
+                  tc_commit(tfull_bar);
+                  ++clamp_idx;
+                }
+                j = 0;
+                ++acc;
+              }
             }
           }
           if (!ok) break;

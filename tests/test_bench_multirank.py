@@ -47,7 +47,7 @@ def test_reference_arm_prints_on_rank0_only(capsys, monkeypatch):
     import bench
 
     class A:
-        size, steps, warmup, gpus, no_merge, layout = 256, 1, 0, 2, False, "dgrad"
+        size, steps, warmup, gpus, no_merge, layout, acc_tile, acc_bits = 256, 1, 0, 2, False, "dgrad", 32, 8
 
     monkeypatch.setenv("RANK", "1")
     bench.run_reference(A)
