@@ -31,8 +31,9 @@
  *     ran out) are recorded in *dev_status (device int32, sticky maximum of
  *     hdqt_status_t values; the caller zeroes it and reads it after a
  *     synchronise).  dev_status may be NULL (such errors are then dropped).
- *   - Alignment: src / out pointers 16 bytes; code buffers and workspaces
- *     128 bytes.
+ *   - Alignment: fp32 sources and outputs 4 bytes (16 bytes, with leading
+ *     dimensions that are multiples of 4, select the vector paths); code
+ *     buffers and workspaces 128 bytes (256 for the three-GEMM calls).
  *   - Code layout: int8 lanes, row-major [rows, K_pad] with the contraction
  *     index contiguous, K_pad = hdqt_padded_k(K, had_block); padded entries are
  *     codes of zero-padded source entries.
@@ -115,7 +116,10 @@ const char* hdqt_status_string(hdqt_status_t s);
  *
  * src: fp32, logical shape [rows, K]; element (r, k) is src[r*ld_row + k*ld_k].
  *      Exactly one of ld_row, ld_k must be 1 (K contiguous, or K strided with
- *      the row index contiguous); the other must be a multiple of 4.
+ *      the row index contiguous); the other must cover the contiguous extent
+ *      (ld_row >= K, resp. ld_k >= rows).  With K contiguous, a 16-byte aligned
+ *      src and ld_row % 4 == 0 select 128-bit loads; anything else still works
+ *      through scalar loads.
  * Non-finite values set HDQT_ERR_NONFINITE in *dev_status.
  */
 hdqt_status_t hdqt_absmax_hadamard(const float* src, int64_t rows, int64_t K,
@@ -201,7 +205,9 @@ hdqt_status_t hdqt_quantize_hadamard_static(const float* src, int64_t rows, int6
  *     true).  It bounds the tile sums and selects the narrowest exact epilogue; codes that
  *     break the promise give undefined results.
  * step_a, step_b: device scalars written by hdqt_quantize_hadamard.
- * out   : fp32 [M, ld_out] row-major, ld_out >= N.
+ * out   : fp32 [M, ld_out] row-major, ld_out >= N.  While the call runs, `out` may hold
+ *     intermediate integer partial sums (long contractions widen their 16-bit lane sums
+ *     through it); it holds the fp32 result when the kernel has finished.
  * S_out : optional int32 [M, N] (dense): the integer sums S.
  * tiles_out: optional int8/int16 debug output, see `tiles_elem_bytes`: [T, M, N]
  *     per-tile accumulator contents c_t; forces every tile through the clamp path.
