@@ -7,10 +7,10 @@
 //   S        = sum_t c_t                                                   int32 registers
 //   out      = fp32(S) * fp32(step_a*step_b*2^r / n_h)
 //
-// One CTA owns a 128 x 256 output block.  Warp 0 feeds a 4-stage shared-memory ring with TMA
-// (128-byte swizzled rows = 4 tiles of 32 k per stage), warp 1 issues the MMAs into two TMEM
-// accumulators of 256 columns, warps 2..17 drain the accumulators (tcgen05.ld), apply the
-// accumulator quantisation per tile and keep the wide sums in registers.
+// Output blocks are 128 x 256; persistent CTAs (one per SM) walk over them.  Warp 0 feeds a 4-stage
+// shared-memory ring with TMA (128-byte swizzled rows = 4 tiles of 32 k per stage), warp 1 issues the
+// MMAs into two TMEM accumulators of 256 columns, 8 epilogue warps drain the accumulators (tcgen05.ld),
+// apply the accumulator quantisation per tile and keep the wide sums in registers.
 // Tiles that provably cannot clamp (Cauchy-Schwarz bound from per-tile code norms) may be
 // accumulated together in TMEM: the clamp is the identity there, so the integers are unchanged.
 // Every wait is bounded; when one runs out the CTA records HDQT_ERR_TIMEOUT and leaves.
@@ -30,15 +30,19 @@ constexpr int STAGES = 4;
 constexpr int A_STAGE = BM * BKB;              // 16 KB
 constexpr int B_STAGE = BN * BKB;              // 32 KB
 constexpr int STAGE_BYTES = A_STAGE + B_STAGE; // 48 KB
-constexpr int NUM_EPI_WARPS = 16;              // 4 per TMEM lane quarter, 64 accumulator columns each
+constexpr int NUM_EPI_WARPS = 8;               // 2 per TMEM lane quarter, 128 accumulator columns each
 constexpr int EPI_COLS = BN / (NUM_EPI_WARPS / 4);
-constexpr int GEMM_THREADS = 32 * (2 + NUM_EPI_WARPS);
+constexpr int GEMM_THREADS = 32 * (3 + NUM_EPI_WARPS);   // + TMA producer, MMA issuer, certificate builder
 constexpr int TMEM_COLS = 512;
-constexpr int MAX_CERT_WORDS = 512;            // certificate bitmask: up to 16384 accumulator tiles
-constexpr int STAGE_OUT_ROW = EPI_COLS + 4;     // floats per staged output row (+4: conflict-free float4 rows)
-constexpr int STAGE_OUT_WARP = 32 * STAGE_OUT_ROW;   // floats per epilogue warp (32 rows x 64 columns)
-static_assert(NUM_EPI_WARPS * STAGE_OUT_WARP * 4 <= STAGES * STAGE_BYTES, "output staging must fit the operand ring");
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 4 * MAX_CERT_WORDS;
+constexpr int MAX_CERT_WORDS = 256;            // certificate bitmask: up to 8192 accumulator tiles
+constexpr int OUT_STAGE_WARP = 32 * 16 * 4;    // per epilogue warp: a 32-row x 16-column fp32 box for the store transpose
+constexpr int TILE_INFO_BYTES = 4 * MAX_CERT_WORDS + 16;
+// the dynamic shared-memory window is declared 1024-byte aligned (checked in the kernel), so no slack is kept
+// offset of the store boxes (128-byte aligned)
+constexpr int OUT_STAGE_OFF = (STAGES * STAGE_BYTES + 256 /*barriers*/ + 2 * TILE_INFO_BYTES + 127) / 128 * 128;
+constexpr int SMEM_BYTES = OUT_STAGE_OFF + NUM_EPI_WARPS * OUT_STAGE_WARP;
+static_assert(OUT_STAGE_WARP % 128 == 0, "store boxes must stay 128-byte aligned");
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
 // instruction descriptor: D = s32, A = B = signed 8-bit, both K-major, N = 256, M = 128
 constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
@@ -226,6 +230,16 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
                :                                                                                        \
                : "memory")
 
+#define HDQT_TMEM_WAIT32(v)                                                                             \
+  asm volatile("tcgen05.wait::ld.sync.aligned;"                                                         \
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]),    \
+                 "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), \
+                 "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]),          \
+                 "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]),          \
+                 "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])           \
+               :                                                                                        \
+               : "memory")
+
 #define HDQT_TMEM_LD16(taddr, v)                                                                        \
   asm volatile(                                                                                         \
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "                                                         \
@@ -235,6 +249,18 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
         "=r"(v[15])                                                                                     \
       : "r"(taddr)                                                                                      \
       : "memory")
+
+// packed (two columns per register) load of half of a warp's columns, and the matching wait
+#define HDQT_LD_HALF_PACK(taddr, v)                                    \
+  do {                                                                 \
+    if constexpr (EPI_COLS / 4 == 32) { HDQT_TMEM_LD32_PACK16(taddr, v); } \
+    else { HDQT_TMEM_LD16_PACK16(taddr, v); }                          \
+  } while (0)
+#define HDQT_WAIT_HALF(v)                                              \
+  do {                                                                 \
+    if constexpr (EPI_COLS / 4 == 32) { HDQT_TMEM_WAIT32(v); }         \
+    else { HDQT_TMEM_WAIT16(v); }                                      \
+  } while (0)
 
 // accumulator quantisation of one exact tile sum
 template <bool kShift>
@@ -249,12 +275,9 @@ __device__ __forceinline__ int acc_quant(int P, int r, int lo, int hi) {
 // Writes 4 consecutive output columns of one row: the final fp32 values (and optionally the integer
 // sums), or - for an intermediate widening of the packed sums - the int32 partial sums, which are
 // parked in the output buffer itself until the final pass reads them back.
-// In the final pass of the vector path the fp32 values go to `stage` (this thread's row of the warp's
-// shared-memory staging block) instead, and the warp copies the block out row by row afterwards, so
-// that global stores are 256 contiguous bytes per half-warp rather than 16 bytes per row.
 template <bool kFinal>
 __device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t gn, int (&s)[4], bool have_prev,
-                                      bool vec, float scale, float* stage = nullptr) {
+                                      bool vec, float scale) {
   float* orow = p.out + gm * p.ld_out + gn;
   if (vec) {
     if (have_prev) {
@@ -267,7 +290,7 @@ __device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t g
       o.y = __fmul_rn((float)s[1], scale);
       o.z = __fmul_rn((float)s[2], scale);
       o.w = __fmul_rn((float)s[3], scale);
-      *reinterpret_cast<float4*>(stage != nullptr ? stage : orow) = o;
+      *reinterpret_cast<float4*>(orow) = o;
     } else {
       *reinterpret_cast<int4*>(orow) = make_int4(s[0], s[1], s[2], s[3]);
     }
@@ -289,48 +312,304 @@ __device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t g
   }
 }
 
+// ---- epilogue of one output block, as separate functions ---------------------------------------
+// Each variant keeps its own register-resident state (sums, load buffers); keeping them out of the
+// kernel body lets the compiler allocate registers per variant instead of for their union.
+
+struct EpiCtx {               // constants of one epilogue warp
+  uint32_t lane_addr;         // TMEM address of this warp's lane quarter and column group in accumulator 0
+  uint32_t bar_tfull;         // [2] accumulator ready
+  uint32_t bar_tempty;        // [2] accumulator drained
+  volatile int* abort_flag;
+  float* box;                 // this warp's 32 x 16 fp32 staging box in shared memory
+  int q, grp, lane;
+};
+
+struct BlockJob {             // one output block as seen by the epilogue
+  int m0, n0;
+  int n_clamp_tiles;          // accumulator tiles that arrive one by one for the clamp path
+  int n_merged;               // accumulator tiles merged in accumulator 0
+  int merging;                // clamp tiles use accumulator 1 only (else they alternate 0 / 1)
+};
+
+__device__ __forceinline__ float dequant_scale(const GemmParams& p) {
+  return (float)((double)__ldg(p.step_a) * (double)__ldg(p.step_b) * (double)(1u << p.acc_shift) /
+                 (double)p.had_block);
+}
+
+// Final integer sums of columns [16c, 16c+16) of this thread's row -> fp32 output.
+// Staged path: the warp's 32 x 16 block is transposed through a 2 KB shared-memory box so that every
+// store instruction writes 8 rows x 64 contiguous bytes (whole sectors) instead of 32 rows x 16 bytes;
+// stores are fire-and-forget, so the box can be reused as soon as the warp has read it back.
+__device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e, const BlockJob& job, int c,
+                                            int (&val)[16], bool parked, float scale) {
+  const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
+  const int64_t gn = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16;
+  const bool staged = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+                      (gn + 16 <= p.N);    // warp-uniform
+  if (staged) {
+    if (gm < p.M && (parked || p.S_out != nullptr)) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        if (parked) val[i] += __float_as_int(p.out[gm * p.ld_out + gn + i]);
+        if (p.S_out != nullptr) p.S_out[gm * p.N + gn + i] = val[i];
+      }
+    }
+    // row r of the box starts at r*16 floats; the four float4 of a row are rotated by (r >> 1) & 3 so
+    // that neither the row-wise writes nor the read-back hit a shared-memory bank twice
+    float4* dst = reinterpret_cast<float4*>(e.box + e.lane * 16);
+    const int rot = (e.lane >> 1) & 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      dst[(i + rot) & 3] = make_float4(__fmul_rn((float)val[4 * i], scale), __fmul_rn((float)val[4 * i + 1], scale),
+                                       __fmul_rn((float)val[4 * i + 2], scale), __fmul_rn((float)val[4 * i + 3], scale));
+    }
+    __syncwarp();
+    const int sub = e.lane >> 2, quad = e.lane & 3;       // 8 rows per instruction, 4 lanes per row
+#pragma unroll
+    for (int rr = 0; rr < 32; rr += 8) {
+      const int rloc = rr + sub;
+      const float4 v = *reinterpret_cast<const float4*>(e.box + rloc * 16 + ((quad + ((rloc >> 1) & 3)) & 3) * 4);
+      const int64_t grow = (int64_t)job.m0 + e.q * 32 + rloc;
+      if (grow < p.M) *reinterpret_cast<float4*>(p.out + grow * p.ld_out + gn + quad * 4) = v;
+    }
+    __syncwarp();
+  } else if (gm < p.M) {
+#pragma unroll
+    for (int i = 0; i < 16; i += 4) {
+      int s4[4] = {val[i], val[i + 1], val[i + 2], val[i + 3]};
+      emit4<true>(p, gm, gn + i, s4, parked, false, scale);
+    }
+  }
+}
+
+__device__ __forceinline__ void release_accumulator(const EpiCtx& e, int buf, uint32_t* drains) {
+  tc_fence_before();
+  __syncwarp();
+  if (e.lane == 0) mbar_arrive(e.bar_tempty + 8 * buf);
+  ++drains[buf];
+}
+
+// Whole block merged (the common case on heavy-tailed operands): no per-tile sums exist, so the registers
+// take the complete accumulator row at once and the accumulator goes back to the MMA issuer before any
+// conversion or store work.
+__device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+  if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+  tc_fence_after();
+  const float scale = dequant_scale(p);
+  uint32_t mv[EPI_COLS];
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) HDQT_TMEM_LD16(e.lane_addr + c * 16, (mv + c * 16));
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) HDQT_TMEM_WAIT16((mv + c * 16));
+  release_accumulator(e, 0, drains);
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) {
+    int val[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) val[i] = (int)mv[c * 16 + i];
+    store_chunk(p, e, job, c, val, false, scale);
+  }
+  return true;
+}
+
+// 16-bit-lane path: tile sums fit int16, b_a <= 8, r = 0.  TMEM is read with two columns packed per
+// register (low half = even column); c - lo = relu(min(P - lo, hi - lo)) per lane in one instruction;
+// sums stay unsigned 16-bit lanes and are widened through the output buffer every flush_every tiles.
+__device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+  uint32_t S[EPI_COLS / 2];
+#pragma unroll
+  for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+  const uint32_t off = (uint32_t)(-p.lo);                    // c - lo lies in [0, hi - lo]
+  const uint32_t off2 = off | (off << 16);
+  const uint32_t rng2 = (uint32_t)(p.hi - p.lo) | ((uint32_t)(p.hi - p.lo) << 16);
+  int n_in_S = 0;
+  bool parked = false;   // int32 partial sums are parked in the output buffer
+  // Half of the warp's columns at a time through one load buffer; the other epilogue warp of the
+  // scheduler covers the load latency.
+  for (int ci = 0; ci < job.n_clamp_tiles; ++ci) {
+    const int buf = job.merging ? 1 : (ci & 1);
+    if (!mbar_wait(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+    uint32_t v[EPI_COLS / 4];
+    HDQT_LD_HALF_PACK(e.lane_addr + buf * BN, v);
+    HDQT_WAIT_HALF(v);
+#pragma unroll
+    for (int i = 0; i < EPI_COLS / 4; ++i) S[i] += __viaddmin_s16x2_relu(v[i], off2, rng2);
+    HDQT_LD_HALF_PACK(e.lane_addr + buf * BN + EPI_COLS / 2, v);
+    HDQT_WAIT_HALF(v);                                                 // the buffer is free
+    release_accumulator(e, buf, drains);
+#pragma unroll
+    for (int i = 0; i < EPI_COLS / 4; ++i) S[EPI_COLS / 4 + i] += __viaddmin_s16x2_relu(v[i], off2, rng2);
+    if (++n_in_S == p.flush_every && ci + 1 < job.n_clamp_tiles) {
+      // widen: park int32 partial sums in the output buffer
+      const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
+      const int64_t gn0 = (int64_t)job.n0 + e.grp * EPI_COLS;
+      const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+                       (gn0 + EPI_COLS <= p.N);
+      if (gm < p.M) {
+#pragma unroll
+        for (int i = 0; i < EPI_COLS / 2; i += 2) {
+          int s4[4];
+          s4[0] = (int)(S[i] & 0xFFFFu) - (int)off * n_in_S;
+          s4[1] = (int)(S[i] >> 16) - (int)off * n_in_S;
+          s4[2] = (int)(S[i + 1] & 0xFFFFu) - (int)off * n_in_S;
+          s4[3] = (int)(S[i + 1] >> 16) - (int)off * n_in_S;
+          emit4<false>(p, gm, gn0 + 2 * i, s4, parked, vec, 0.0f);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+      n_in_S = 0;
+      parked = true;
+    }
+  }
+  if (job.n_merged > 0) {
+    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+  }
+  const float scale = dequant_scale(p);
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) {
+    uint32_t mv[16];
+    if (job.n_merged > 0) {   // uniform
+      HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
+      HDQT_TMEM_WAIT16(mv);
+      // the last of the merged accumulator is in registers: hand it back to the MMA issuer
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drains);
+    }
+    int val[16];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t sp = S[c * 8 + i];
+      val[2 * i] = (int)(sp & 0xFFFFu) - (int)off * n_in_S;
+      val[2 * i + 1] = (int)(sp >> 16) - (int)off * n_in_S;
+      if (job.n_merged > 0) {
+        val[2 * i] += (int)mv[2 * i];
+        val[2 * i + 1] += (int)mv[2 * i + 1];
+      }
+    }
+    store_chunk(p, e, job, c, val, parked, scale);
+  }
+  return true;
+}
+
+// 32-bit path: one register per accumulator element, any b_a and shift r, optional per-tile debug output.
+template <bool kShift, bool kTilesOut>
+__device__ __forceinline__ bool epilogue_wide(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+  int S[EPI_COLS];
+#pragma unroll
+  for (int i = 0; i < EPI_COLS; ++i) S[i] = 0;
+  const int r = p.acc_shift, lo = p.lo, hi = p.hi;
+  for (int ci = 0; ci < job.n_clamp_tiles; ++ci) {
+    const int buf = job.merging ? 1 : (ci & 1);
+    if (!mbar_wait(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+#pragma unroll
+    for (int c = 0; c < EPI_COLS / 16; ++c) {
+      uint32_t v[16];
+      HDQT_TMEM_LD16(e.lane_addr + buf * BN + c * 16, v);
+      HDQT_TMEM_WAIT16(v);
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, buf, drains);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int ct = acc_quant<kShift>((int)v[i], r, lo, hi);
+        S[c * 16 + i] += ct;
+        if (kTilesOut) {
+          const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
+          const int64_t n = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16 + i;
+          if (gm < p.M && n < p.N) {
+            const int64_t o = ((int64_t)ci * p.M + gm) * p.N + n;
+            if (p.tiles_elem_bytes == 1) reinterpret_cast<int8_t*>(p.tiles_out)[o] = (int8_t)ct;
+            else reinterpret_cast<int16_t*>(p.tiles_out)[o] = (int16_t)ct;
+          }
+        }
+      }
+    }
+  }
+  if (job.n_merged > 0) {
+    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+  }
+  const float scale = dequant_scale(p);
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) {
+    int val[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) val[i] = S[c * 16 + i];
+    if (job.n_merged > 0) {   // uniform
+      uint32_t mv[16];
+      HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
+      HDQT_TMEM_WAIT16(mv);
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drains);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) val[i] += (int)mv[i];
+    }
+    store_chunk(p, e, job, c, val, false, scale);
+  }
+  return true;
+}
+
 // ---- the kernel -----------------------------------------------------------------------------
+// Persistent: one CTA per SM walks over output blocks (block index = blockIdx.x + i*gridDim.x), so that the
+// TMA producer runs ahead into the next block while the epilogue warps drain the previous one, and the
+// per-block fixed costs (TMEM allocation, barrier set-up, pipeline fill) are paid once.
+//
+// Warp roles: 0 = TMA producer, 1 = MMA issuer, 2 = certificate builder (clamp-free tile bitmask of the
+// next block, from the tile norms), 3..10 = epilogue (TMEM lane quarter = warp % 4, 128 columns each;
+// 11 warps leave each thread 168 registers: the sums of 128 columns plus a load buffer fit without spills).
+//
 // kPacked: the per-tile sums fit 16 bits and b_a <= 8, r = 0: TMEM is read with two columns packed
 //          per register, clamp and add work on 16-bit lane pairs (half the ALU work per element).
 // otherwise: one 32-bit register per accumulator element, any b_a and r.
 
+struct TileInfo {                       // what the certificate warp publishes per output block
+  uint32_t mask[MAX_CERT_WORDS];        // bit a: accumulator tile a provably cannot clamp
+  int32_t n_uncert;                     // accumulator tiles without a certificate
+  int32_t pad[3];
+};
+static_assert(sizeof(TileInfo) == TILE_INFO_BYTES, "TileInfo layout");
+
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tile_m, int& tile_n) {
+  // grouped order: co-resident CTAs form a roughly square patch (16 row blocks x ~9 column blocks on
+  // 148 SMs), so both operands' panels are shared through L2
+  constexpr int GROUP_M = 16;
+  const int per_group = GROUP_M * tiles_n;
+  const int group = t / per_group;
+  const int first_m = group * GROUP_M;
+  const int group_rows = min(tiles_m - first_m, GROUP_M);
+  const int in_group = t - group * per_group;
+  tile_m = first_m + in_group % group_rows;
+  tile_n = in_group / group_rows;
+}
+
 template <bool kPacked, bool kShift, bool kTilesOut>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                     const GemmParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+                     const __grid_constant__ GemmParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
+  uint8_t* smem_al = smem_raw;
+  if (smem_base & 1023u) {   // the 128-byte swizzle needs 1024-byte aligned stages: refuse rather than corrupt
+    if (threadIdx.x == 0) report_status(p.dev_status, HDQT_ERR_CUDA);
+    return;
+  }
   // barrier block behind the stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * STAGE_BYTES);
-  const uint32_t bar_full = smem_u32(bars);             // [STAGES]
-  const uint32_t bar_empty = bar_full + 8 * STAGES;     // [STAGES]
-  const uint32_t bar_tfull = bar_empty + 8 * STAGES;    // [2]
-  const uint32_t bar_tempty = bar_tfull + 16;           // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  const uint32_t bar_full = smem_u32(bars);             // [STAGES]  TMA -> MMA
+  const uint32_t bar_empty = bar_full + 8 * STAGES;     // [STAGES]  MMA -> TMA
+  const uint32_t bar_tfull = bar_empty + 8 * STAGES;    // [2]       MMA -> epilogue (accumulator ready)
+  const uint32_t bar_tempty = bar_tfull + 16;           // [2]       epilogue -> MMA (accumulator drained)
+  const uint32_t bar_ifull = bar_tempty + 16;           // [2]       certificate warp -> MMA, epilogue
+  const uint32_t bar_iempty = bar_ifull + 16;           // [2]       MMA, epilogue -> certificate warp
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* s_uncert = reinterpret_cast<int*>(tmem_slot + 2);
-  uint32_t* cert_mask = reinterpret_cast<uint32_t*>(smem_al + STAGES * STAGE_BYTES + 256);
+  TileInfo* tile_info = reinterpret_cast<TileInfo*>(smem_al + STAGES * STAGE_BYTES + 256);   // [2]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  // 1-D grid over output blocks, ordered so that co-resident CTAs form a roughly square patch
-  // (16 row blocks x ~9 column blocks on 148 SMs): both operands' panels are then shared through L2
   const int tiles_m = (int)((p.M + BM - 1) / BM), tiles_n = (int)((p.N + BN - 1) / BN);
-  int tile_m, tile_n;
-  {
-    constexpr int GROUP_M = 16;
-    const int t = blockIdx.x;
-    const int per_group = GROUP_M * tiles_n;
-    const int group = t / per_group;
-    const int first_m = group * GROUP_M;
-    const int group_rows = min(tiles_m - first_m, GROUP_M);
-    const int in_group = t - group * per_group;
-    tile_m = first_m + in_group % group_rows;
-    tile_n = in_group / group_rows;
-  }
-  const int m0 = tile_m * BM;
-  const int n0 = tile_n * BN;
+  const int num_tiles = tiles_m * tiles_n;
   const int num_kblocks = (p.tiles32 + 3) >> 2;
   const int num_acc = p.num_acc;
 
@@ -342,9 +621,10 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_tfull + 8 * b, 1);
       mbar_init(bar_tempty + 8 * b, NUM_EPI_WARPS);
+      mbar_init(bar_ifull + 8 * b, 1);
+      mbar_init(bar_iempty + 8 * b, NUM_EPI_WARPS + 1);
     }
     *abort_flag = 0;
-    *s_uncert = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -359,70 +639,87 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // ---- which accumulator tiles provably cannot clamp (Cauchy-Schwarz on the tile norms) ----
-  // bit a of cert_mask is set iff every 32-wide sub-tile of accumulator tile a satisfies
-  // max_row ||a||^2 * max_col ||b||^2 <= (hi / tiles_per_acc)^2, so |P| <= hi for the whole block.
-  if (p.merge == 1) {
-    if (warp >= 2) {
-      const int et = threadIdx.x - 64;
-      const int64_t T = p.tiles32;
-      const int32_t* na = p.norms_a + (int64_t)tile_m * T;
-      const int64_t nb_blk = (int64_t)tile_n * 2;
-      const int32_t* nb0 = p.norms_b + nb_blk * T;
-      const bool has1 = (nb_blk + 1) * 128 < p.N;
-      const int32_t* nb1 = nb0 + T;
-      int my_uncert = 0;
-      const int acc_round = (num_acc + 31) & ~31;
-      for (int a = et; a < acc_round; a += 32 * NUM_EPI_WARPS) {
-        bool cert = false;
-        if (a < num_acc) {
-          cert = true;
-          const int t0 = a * p.tiles_per_acc;
-          const int t1 = min(p.tiles32, t0 + p.tiles_per_acc);
-          for (int t = t0; t < t1; ++t) {
-            const int64_t a2 = __ldg(na + t);
-            int64_t b2 = __ldg(nb0 + t);
-            if (has1) b2 = max(b2, (int64_t)__ldg(nb1 + t));
-            cert = cert && (a2 * b2 <= p.cert_thr_sq);
-          }
-          my_uncert += cert ? 0 : 1;
-        }
-        const uint32_t bits = __ballot_sync(0xFFFFFFFFu, cert);
-        if (lane == 0) cert_mask[a >> 5] = bits;
-      }
-      my_uncert = __reduce_add_sync(0xFFFFFFFFu, my_uncert);
-      if (lane == 0 && my_uncert) atomicAdd(s_uncert, my_uncert);
-    }
-    __syncthreads();
-  }
-  const int n_uncert = (p.merge == 2) ? 0 : *s_uncert;
-  // merge in this CTA only when few tiles need the clamp path (it is single-buffered when merging)
-  const bool merging = (p.merge == 2) ||
-                       (p.merge == 1 && (int64_t)n_uncert * 256 <= (int64_t)p.merge_max_uncert_256 * num_acc);
-  const int n_clamp_tiles = merging ? n_uncert : num_acc;
-  const int n_merged = merging ? num_acc - n_uncert : 0;
+  // A block merges its certified tiles only when few tiles need the clamp path (that path is
+  // single-buffered while merging).
+  auto block_merges = [&](int n_uncert) {
+    return (p.merge == 2) ||
+           (p.merge == 1 && (int64_t)n_uncert * 256 <= (int64_t)p.merge_max_uncert_256 * num_acc);
+  };
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < num_kblocks; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t par = ((kb / STAGES) & 1) ^ 1;
-        if (!mbar_wait(bar_empty + 8 * s, par, abort_flag)) break;
-        mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
-        const uint32_t a_dst = smem_base + s * STAGE_BYTES;
-        tma_load_2d(a_dst, &map_a, kb * BKB, m0, bar_full + 8 * s);
-        tma_load_2d(a_dst + A_STAGE, &map_b, kb * BKB, n0, bar_full + 8 * s);
-        issued = kb + 1;
+      uint32_t it = 0;   // k-blocks issued so far, over all output blocks
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int tile_m, tile_n;
+        tile_coords(tile, tiles_m, tiles_n, tile_m, tile_n);
+        for (int kb = 0; kb < num_kblocks; ++kb, ++it) {
+          const uint32_t s = it % STAGES;
+          const uint32_t par = ((it / STAGES) & 1u) ^ 1u;
+          if (!mbar_wait(bar_empty + 8 * s, par, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
+          const uint32_t a_dst = smem_base + s * STAGE_BYTES;
+          tma_load_2d(a_dst, &map_a, kb * BKB, tile_m * BM, bar_full + 8 * s);
+          tma_load_2d(a_dst + A_STAGE, &map_b, kb * BKB, tile_n * BN, bar_full + 8 * s);
+        }
       }
       if (*abort_flag) {
         // let the copies that are still in flight land before the CTA gives its memory back
-        for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
-          const uint32_t bar = bar_full + 8 * (kb % STAGES);
-          const uint32_t par = (kb / STAGES) & 1;
+        for (uint32_t k = (it > STAGES ? it - STAGES : 0u); k < it; ++k) {
+          const uint32_t bar = bar_full + 8 * (k % STAGES);
+          const uint32_t par = (k / STAGES) & 1u;
           for (int i = 0; i < (1 << 16) && !mbar_try_wait(bar, par); ++i) __nanosleep(256);
         }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------ certificate builder ------------------------
+    // bit a is set iff every 32-wide sub-tile of accumulator tile a satisfies
+    // max_row ||a||^2 * max_col ||b||^2 <= (hi / tiles_per_acc)^2, so |P| <= hi for the whole block
+    // (Cauchy-Schwarz) and the clamp is the identity there.
+    if (p.merge == 1) {
+      int ti = 0;
+      for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++ti) {
+        const int slot = ti & 1;
+        if (!mbar_wait_yield<128>(bar_iempty + 8 * slot, (((uint32_t)ti >> 1) & 1u) ^ 1u, abort_flag)) break;
+        int tile_m, tile_n;
+        tile_coords(tile, tiles_m, tiles_n, tile_m, tile_n);
+        const int64_t T = p.tiles32;
+        const int32_t* na = p.norms_a + (int64_t)tile_m * T;
+        const int64_t nb_blk = (int64_t)tile_n * 2;
+        const int32_t* nb0 = p.norms_b + nb_blk * T;
+        const bool has1 = (nb_blk + 1) * 128 < p.N;
+        const int32_t* nb1 = nb0 + T;
+        TileInfo& info = tile_info[slot];
+        int uncert = 0;
+        const int acc_round = (num_acc + 31) & ~31;
+        for (int a = lane; a < acc_round; a += 32) {
+          bool cert = false;
+          if (a < num_acc) {
+            cert = true;
+            const int t0 = a * p.tiles_per_acc;
+            const int t1 = min(p.tiles32, t0 + p.tiles_per_acc);
+            for (int t = t0; t < t1; ++t) {
+              const int64_t a2 = __ldg(na + t);
+              int64_t b2 = __ldg(nb0 + t);
+              if (has1) b2 = max(b2, (int64_t)__ldg(nb1 + t));
+              cert = cert && (a2 * b2 <= p.cert_thr_sq);
+            }
+          }
+          const uint32_t bits = __ballot_sync(0xFFFFFFFFu, cert);
+          if (lane == 0) {
+            info.mask[a >> 5] = bits;
+            const int valid = min(32, num_acc - a);
+            uncert += valid - __popc(valid == 32 ? bits : (bits & ((1u << valid) - 1u)));
+          }
+        }
+        if (lane == 0) {
+          info.n_uncert = uncert;
+          __threadfence_block();
+          mbar_arrive(bar_ifull + 8 * slot);
+        }
+        __syncwarp();
       }
     }
   } else if (warp == 1) {
@@ -434,41 +731,54 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       // the next stage's barrier polled ahead; only stages with clamp tiles take the per-tile code.
       const uint64_t desc_a0 = make_smem_desc(smem_base);
       const uint64_t desc_b0 = make_smem_desc(smem_base + A_STAGE);
-      int s = 0;                 // smem stage
+      uint32_t s = 0;            // smem stage
       uint32_t full_par = 0;     // parity of the stage's next "full" phase
-      int j = 0;                 // position inside the current accumulator tile
-      int acc = 0;               // accumulator tile index
-      int clamp_idx = 0;         // index among the tiles that take the clamp path
-      bool cert = (p.merge == 2);
-      uint32_t merged_started = 0;
-      uint32_t d_tmem = tmem_base;
-      uint32_t tfull_bar = bar_tfull;
+      uint32_t fills[2] = {0u, 0u};   // how many times each TMEM accumulator has been handed to the epilogue
       uint64_t desc_a = desc_a0, desc_b = desc_b0;
       bool ok = true;
       const int tiles32 = p.tiles32, tpa = p.tiles_per_acc;
-      const bool nibble_ok = (p.merge == 2) || (merging && tpa == 1);
-      bool ready = mbar_test_wait(bar_full, 0u);
-      for (int kb = 0; kb < num_kblocks; ++kb) {
-        if (!ready && !mbar_wait(bar_full + 8 * s, full_par, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        // poll the next stage now; the answer is needed only after this stage's MMAs
-        const int s_next = (s + 1 == STAGES) ? 0 : s + 1;
-        const uint32_t par_next = (s + 1 == STAGES) ? (full_par ^ 1u) : full_par;
-        const int kt0 = kb * 4;
-        uint32_t nib = 0;
-        if (p.merge == 2) nib = 0xFu;
-        else if (nibble_ok) nib = (cert_mask[kb >> 3] >> ((kb & 7) * 4)) & 0xFu;
-        if (nib == 0xFu && kt0 + 4 <= tiles32) {
-          tc_mma_i8(tmem_base, desc_a, desc_b, merged_started);
-          tc_mma_i8(tmem_base, desc_a + 2, desc_b + 2, 1u);
-          tc_mma_i8(tmem_base, desc_a + 4, desc_b + 4, 1u);
-          tc_mma_i8(tmem_base, desc_a + 6, desc_b + 6, 1u);
-          merged_started = 1u;
-          acc += 4;    // only meaningful (and only used) when tiles_per_acc == 1
-        } else {
-          if (tpa < 4) {
-            // short accumulator tiles: one MMA per pass keeps this thread's path between a released
-            // accumulator and the next MMA as short as possible (it is on the critical chain of every tile)
+      bool ready = false;
+      int ti = 0;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ti) {
+        const int slot = ti & 1;
+        int n_uncert = (p.merge == 2) ? 0 : num_acc;
+        if (p.merge == 1) {
+          if (!mbar_wait(bar_ifull + 8 * slot, ((uint32_t)ti >> 1) & 1u, abort_flag)) { ok = false; break; }
+          n_uncert = *reinterpret_cast<volatile int32_t*>(&tile_info[slot].n_uncert);
+        }
+        const bool merging = block_merges(n_uncert);
+        const int n_merged = merging ? num_acc - n_uncert : 0;
+        const uint32_t* cert_mask = tile_info[slot].mask;
+        const bool nibble_ok = (p.merge == 2) || (merging && p.merge == 1 && tpa == 1);
+        int j = 0;                 // position inside the current accumulator tile
+        int acc = 0;               // accumulator tile index
+        int clamp_idx = 0;         // index among this block's tiles that take the clamp path
+        bool cert = (p.merge == 2);
+        uint32_t merged_started = 0;
+        uint32_t d_tmem = tmem_base;
+        int cur_buf = 0;
+        for (int kb = 0; kb < num_kblocks; ++kb) {
+          if (!ready && !mbar_wait(bar_full + 8 * s, full_par, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t s_next = (s + 1 == STAGES) ? 0u : s + 1;
+          const uint32_t par_next = (s + 1 == STAGES) ? (full_par ^ 1u) : full_par;
+          const int kt0 = kb * 4;
+          uint32_t nib = 0;
+          if (p.merge == 2) nib = 0xFu;
+          else if (nibble_ok) nib = (cert_mask[kb >> 3] >> ((kb & 7) * 4)) & 0xFu;
+          if (nib == 0xFu && kt0 + 4 <= tiles32) {
+            if (!merged_started) {
+              // the merged accumulator (buffer 0) must have been drained by the previous user
+              if (!mbar_wait(bar_tempty, (fills[0] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+            }
+            tc_mma_i8(tmem_base, desc_a, desc_b, merged_started);
+            tc_mma_i8(tmem_base, desc_a + 2, desc_b + 2, 1u);
+            tc_mma_i8(tmem_base, desc_a + 4, desc_b + 4, 1u);
+            tc_mma_i8(tmem_base, desc_a + 6, desc_b + 6, 1u);
+            merged_started = 1u;
+            acc += 4;    // only meaningful (and only used) when tiles_per_acc == 1
+          } else {
             const int kt1 = min(tiles32, kt0 + 4);
             for (int kt = kt0; kt < kt1; ++kt) {
               if (j == 0) {
@@ -477,275 +787,97 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 } else if (merging) {
                   cert = (cert_mask[acc >> 5] >> (acc & 31)) & 1u;
                 }
-                if (cert) {
-                  d_tmem = tmem_base;                      // merged tiles accumulate in buffer 0
-                } else {
-                  // clamp tiles: buffer 1 when merging, else alternate 0 / 1
-                  const int buf = merging ? 1 : (clamp_idx & 1);
-                  const uint32_t use = merging ? (uint32_t)clamp_idx : (uint32_t)(clamp_idx >> 1);
-                  if (!mbar_wait(bar_tempty + 8 * buf, (use & 1) ^ 1, abort_flag)) { ok = false; break; }
+                // merged tiles accumulate in buffer 0; clamp tiles use buffer 1 when merging, else 0 / 1
+                cur_buf = cert ? 0 : (merging ? 1 : (clamp_idx & 1));
+                if (!cert || !merged_started) {
+                  if (!mbar_wait(bar_tempty + 8 * cur_buf, (fills[cur_buf] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                   tc_fence_after();
-                  d_tmem = tmem_base + buf * BN;
-                  tfull_bar = bar_tfull + 8 * buf;
                 }
+                d_tmem = tmem_base + cur_buf * BN;
               }
-              const uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
-              tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, cert ? merged_started : (uint32_t)(j != 0));
+              uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
+              uint32_t accumulate = cert ? merged_started : (uint32_t)(j != 0);
+              tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, accumulate);
+              if (tpa >= 4) {
+                // long accumulator tiles: the rest of this stage's K tiles that belong to the same
+                // accumulator tile go out back to back (bookkeeping between MMAs is dead tensor time)
+                const int extra = min(kt1 - kt, tpa - j) - 1;
+                for (int i = 0; i < extra; ++i) {
+                  sub2 += 2;
+                  tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, 1u);
+                }
+                kt += extra;
+                j += extra;
+              }
               if (cert) merged_started = 1u;
               if (++j == tpa || kt == tiles32 - 1) {
                 if (!cert) {
-                  tc_commit(tfull_bar);
+                  tc_commit(bar_tfull + 8 * cur_buf);
+                  ++fills[cur_buf];
                   ++clamp_idx;
                 }
                 j = 0;
                 ++acc;
               }
             }
-          } else {
-            // long accumulator tiles: the K tiles of this stage that belong to the current accumulator
-            // tile go out back to back
-            const int kt1 = min(tiles32, kt0 + 4);
-            int kt = kt0;
-            while (kt < kt1) {
-              if (j == 0) {
-                if (p.merge == 2) {
-                  cert = true;
-                } else if (merging) {
-                  cert = (cert_mask[acc >> 5] >> (acc & 31)) & 1u;
-                }
-                if (cert) {
-                  d_tmem = tmem_base;                      // merged tiles accumulate in buffer 0
-                } else {
-                  // clamp tiles: buffer 1 when merging, else alternate 0 / 1
-                  const int buf = merging ? 1 : (clamp_idx & 1);
-                  const uint32_t use = merging ? (uint32_t)clamp_idx : (uint32_t)(clamp_idx >> 1);
-                  if (!mbar_wait(bar_tempty + 8 * buf, (use & 1) ^ 1, abort_flag)) { ok = false; break; }
-                  tc_fence_after();
-                  d_tmem = tmem_base + buf * BN;
-                  tfull_bar = bar_tfull + 8 * buf;
-                }
-              }
-              // the K tiles of this stage that belong to the current accumulator tile go out back to back
-              uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
-              uint32_t accumulate = cert ? merged_started : (uint32_t)(j != 0);
-              const int run = min(kt1 - kt, tpa - j);
-              for (int i = 0; i < run; ++i) {
-                tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, accumulate);
-                sub2 += 2;
-                accumulate = 1u;
-              }
-              if (cert) merged_started = 1u;
-              j += run;
-              kt += run;
-              if (j == tpa || kt == tiles32) {
-                if (!cert) {
-                  tc_commit(tfull_bar);
-                  ++clamp_idx;
-                }
-                j = 0;
-                ++acc;
-              }
-            }
+            if (!ok) break;
           }
-          if (!ok) break;
+          tc_commit(bar_empty + 8 * s);
+          ready = mbar_test_wait(bar_full + 8 * s_next, par_next);
+          s = s_next;
+          full_par = par_next;
+          if (s == 0) {
+            desc_a = desc_a0;
+            desc_b = desc_b0;
+          } else {
+            desc_a += (uint64_t)(STAGE_BYTES >> 4);
+            desc_b += (uint64_t)(STAGE_BYTES >> 4);
+          }
         }
-        tc_commit(bar_empty + 8 * s);
-        ready = (kb + 1 < num_kblocks) && mbar_test_wait(bar_full + 8 * s_next, par_next);
-        s = s_next;
-        full_par = par_next;
-        if (s == 0) {
-          desc_a = desc_a0;
-          desc_b = desc_b0;
-        } else {
-          desc_a += (uint64_t)(STAGE_BYTES >> 4);
-          desc_b += (uint64_t)(STAGE_BYTES >> 4);
+        if (!ok) break;
+        if (n_merged > 0) {
+          tc_commit(bar_tfull + 0);
+          ++fills[0];
         }
+        if (p.merge == 1) mbar_arrive(bar_iempty + 8 * slot);
       }
-      if (ok && n_merged > 0) tc_commit(bar_tfull + 0);
     }
   } else {
     // ------------------------------ epilogue warps ----------------------------
-    const int q = warp & 3;                   // TMEM lane quarter this warp may read
-    const int grp = (warp - 2) >> 2;          // which EPI_COLS columns of the accumulator
-    const int row = q * 32 + lane;
-    const int64_t gm = (int64_t)m0 + row;
-    const int64_t gn0 = (int64_t)n0 + grp * EPI_COLS;
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(grp * EPI_COLS);
-    const int r = p.acc_shift, lo = p.lo, hi = p.hi;
-    const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
-                     (gn0 + EPI_COLS <= p.N);
-    bool ok = true;
-    // output staging reuses the operand ring: it is touched only after the last MMA has completed
-    float* stage_warp = reinterpret_cast<float*>(smem_al) + (warp - 2) * STAGE_OUT_WARP;
-    float* stage_row = stage_warp + lane * STAGE_OUT_ROW;
-    // copies the warp's staged 32 x 64 block to global memory, two rows (2 x 256 bytes) per instruction
-    auto copy_out = [&]() {
-      __syncwarp();
-      const int sub_row = lane >> 4, c4 = (lane & 15) * 4;
-#pragma unroll 4
-      for (int rr = 0; rr < 32; rr += 2) {
-        const int rloc = rr + sub_row;
-        const int64_t grow = (int64_t)m0 + q * 32 + rloc;
-        if (grow < p.M) {
-          const float4 v = *reinterpret_cast<const float4*>(stage_warp + rloc * STAGE_OUT_ROW + c4);
-          *reinterpret_cast<float4*>(p.out + grow * p.ld_out + gn0 + c4) = v;
-        }
+    EpiCtx e;
+    e.q = warp & 3;                     // TMEM lane quarter this warp may read
+    e.grp = (warp - 3) >> 2;            // which EPI_COLS columns of the accumulator
+    e.lane = lane;
+    e.lane_addr = tmem_base + ((uint32_t)(e.q * 32) << 16) + (uint32_t)(e.grp * EPI_COLS);
+    e.bar_tfull = bar_tfull;
+    e.bar_tempty = bar_tempty;
+    e.abort_flag = abort_flag;
+    e.box = reinterpret_cast<float*>(smem_al + OUT_STAGE_OFF + (warp - 3) * OUT_STAGE_WARP);
+    uint32_t drains[2] = {0u, 0u};      // how many times this warp has drained each accumulator
+    int ti = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++ti) {
+      const int slot = ti & 1;
+      int n_uncert = (p.merge == 2) ? 0 : num_acc;
+      if (p.merge == 1) {
+        if (!mbar_wait_yield<128>(bar_ifull + 8 * slot, ((uint32_t)ti >> 1) & 1u, abort_flag)) break;
+        n_uncert = *reinterpret_cast<volatile int32_t*>(&tile_info[slot].n_uncert);
       }
-    };
-
-    if (kPacked) {
-      // two columns per register: low half = even column, high half = odd column
-      uint32_t S[EPI_COLS / 2];
-#pragma unroll
-      for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
-      const uint32_t off = (uint32_t)(-lo);                    // c - lo lies in [0, hi - lo]
-      const uint32_t off2 = off | (off << 16);
-      const uint32_t rng2 = (uint32_t)(hi - lo) | ((uint32_t)(hi - lo) << 16);
-      int n_in_S = 0;
-      bool parked = false;   // int32 partial sums are parked in the output buffer
-      // Rolling pipeline over half-tiles (32 columns = 16 packed registers): while one half is clamped
-      // and added, the load of the next half (possibly of the next tile) is in flight.
-      uint32_t v0[EPI_COLS / 4], v1[EPI_COLS / 4];
-      if (n_clamp_tiles > 0) {
-        const int buf = merging ? 1 : 0;
-        if (!mbar_wait(bar_tfull + 8 * buf, 0u, abort_flag)) ok = false;
-        tc_fence_after();
-        if (ok) HDQT_TMEM_LD16_PACK16(lane_addr + buf * BN, v0);
-      }
-      for (int ci = 0; ci < n_clamp_tiles && ok; ++ci) {
-        const int buf = merging ? 1 : (ci & 1);
-        HDQT_TMEM_WAIT16(v0);                                            // first half of tile ci has landed
-        HDQT_TMEM_LD16_PACK16(lane_addr + buf * BN + EPI_COLS / 2, v1);  // second half in flight ...
-#pragma unroll
-        for (int i = 0; i < EPI_COLS / 4; ++i) S[i] += __viaddmin_s16x2_relu(v0[i], off2, rng2);
-        HDQT_TMEM_WAIT16(v1);                                            // ... landed: the buffer is free
-        tc_fence_before();
+      BlockJob job;
+      job.merging = block_merges(n_uncert) ? 1 : 0;
+      job.n_clamp_tiles = job.merging ? n_uncert : num_acc;
+      job.n_merged = job.merging ? num_acc - n_uncert : 0;
+      int tile_m, tile_n;
+      tile_coords(tile, tiles_m, tiles_n, tile_m, tile_n);
+      job.m0 = tile_m * BM;
+      job.n0 = tile_n * BN;
+      bool ok;
+      if (job.n_clamp_tiles == 0 && job.n_merged > 0) ok = epilogue_merged_only(p, e, job, drains);
+      else if (kPacked) ok = epilogue_packed(p, e, job, drains);
+      else ok = epilogue_wide<kShift, kTilesOut>(p, e, job, drains);
+      if (!ok) break;
+      if (p.merge == 1) {
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-        if (ci + 1 < n_clamp_tiles) {
-          const int nbuf = merging ? 1 : ((ci + 1) & 1);
-          const uint32_t use = merging ? (uint32_t)(ci + 1) : (uint32_t)((ci + 1) >> 1);
-          if (!mbar_wait(bar_tfull + 8 * nbuf, use & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          HDQT_TMEM_LD16_PACK16(lane_addr + nbuf * BN, v0);              // first half of the next tile in flight
-        }
-#pragma unroll
-        for (int i = 0; i < EPI_COLS / 4; ++i) S[EPI_COLS / 4 + i] += __viaddmin_s16x2_relu(v1[i], off2, rng2);
-        if (++n_in_S == p.flush_every && ci + 1 < n_clamp_tiles) {
-          // widen: park int32 partial sums in the output buffer
-          if (gm < p.M) {
-#pragma unroll
-            for (int i = 0; i < EPI_COLS / 2; i += 2) {
-              int s4[4];
-              s4[0] = (int)(S[i] & 0xFFFFu) - (int)off * n_in_S;
-              s4[1] = (int)(S[i] >> 16) - (int)off * n_in_S;
-              s4[2] = (int)(S[i + 1] & 0xFFFFu) - (int)off * n_in_S;
-              s4[3] = (int)(S[i + 1] >> 16) - (int)off * n_in_S;
-              emit4<false>(p, gm, gn0 + 2 * i, s4, parked, vec, 0.0f);
-            }
-          }
-#pragma unroll
-          for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
-          n_in_S = 0;
-          parked = true;
-        }
-      }
-      if (ok && n_merged > 0) {
-        ok = mbar_wait_yield<256>(bar_tfull + 0, 0u, abort_flag);
-        tc_fence_after();
-      }
-      if (ok) {
-        const float scale = (float)((double)__ldg(p.step_a) * (double)__ldg(p.step_b) *
-                                    (double)(1u << p.acc_shift) / (double)p.had_block);
-#pragma unroll
-        for (int c = 0; c < EPI_COLS / 16; ++c) {
-          uint32_t mv[16];
-          if (n_merged > 0) {   // uniform
-            HDQT_TMEM_LD16(lane_addr + c * 16, mv);
-            HDQT_TMEM_WAIT16(mv);
-          }
-          if (gm < p.M) {
-#pragma unroll
-            for (int i = 0; i < 8; i += 2) {
-              const uint32_t s0 = S[c * 8 + i], s1 = S[c * 8 + i + 1];
-              int s4[4];
-              s4[0] = (int)(s0 & 0xFFFFu) - (int)off * n_in_S;
-              s4[1] = (int)(s0 >> 16) - (int)off * n_in_S;
-              s4[2] = (int)(s1 & 0xFFFFu) - (int)off * n_in_S;
-              s4[3] = (int)(s1 >> 16) - (int)off * n_in_S;
-              if (n_merged > 0) {
-                s4[0] += (int)mv[2 * i]; s4[1] += (int)mv[2 * i + 1];
-                s4[2] += (int)mv[2 * i + 2]; s4[3] += (int)mv[2 * i + 3];
-              }
-              emit4<true>(p, gm, gn0 + c * 16 + 2 * i, s4, parked, vec, scale,
-                          vec ? stage_row + c * 16 + 2 * i : nullptr);
-            }
-          }
-        }
-        if (vec) copy_out();
-      }
-    } else {
-      int S[EPI_COLS];
-#pragma unroll
-      for (int i = 0; i < EPI_COLS; ++i) S[i] = 0;
-      for (int ci = 0; ci < n_clamp_tiles; ++ci) {
-        const int buf = merging ? 1 : (ci & 1);
-        const uint32_t use = merging ? (uint32_t)ci : (uint32_t)(ci >> 1);
-        if (!mbar_wait(bar_tfull + 8 * buf, use & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < EPI_COLS / 16; ++c) {
-          uint32_t v[16];
-          HDQT_TMEM_LD16(lane_addr + buf * BN + c * 16, v);
-          HDQT_TMEM_WAIT16(v);
-          if (c == EPI_COLS / 16 - 1) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-          }
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int ct = acc_quant<kShift>((int)v[i], r, lo, hi);
-            S[c * 16 + i] += ct;
-            if (kTilesOut) {
-              const int64_t n = gn0 + c * 16 + i;
-              if (gm < p.M && n < p.N) {
-                const int64_t o = ((int64_t)ci * p.M + gm) * p.N + n;
-                if (p.tiles_elem_bytes == 1) reinterpret_cast<int8_t*>(p.tiles_out)[o] = (int8_t)ct;
-                else reinterpret_cast<int16_t*>(p.tiles_out)[o] = (int16_t)ct;
-              }
-            }
-          }
-        }
-      }
-      if (ok && n_merged > 0) {
-        ok = mbar_wait_yield<256>(bar_tfull + 0, 0u, abort_flag);
-        tc_fence_after();
-      }
-      if (ok) {
-        const float scale = (float)((double)__ldg(p.step_a) * (double)__ldg(p.step_b) *
-                                    (double)(1u << p.acc_shift) / (double)p.had_block);
-#pragma unroll
-        for (int c = 0; c < EPI_COLS / 16; ++c) {
-          uint32_t mv[16];
-          if (n_merged > 0) {   // uniform
-            HDQT_TMEM_LD16(lane_addr + c * 16, mv);
-            HDQT_TMEM_WAIT16(mv);
-          }
-          if (gm < p.M) {
-#pragma unroll
-            for (int i = 0; i < 16; i += 4) {
-              int s4[4];
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                s4[j] = S[c * 16 + i + j];
-                if (n_merged > 0) s4[j] += (int)mv[i + j];
-              }
-              emit4<true>(p, gm, gn0 + c * 16 + i, s4, false, vec, scale, vec ? stage_row + c * 16 + i : nullptr);
-            }
-          }
-        }
-        if (vec) copy_out();
+        if (lane == 0) mbar_arrive(bar_iempty + 8 * slot);
       }
     }
   }
@@ -917,7 +1049,8 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
 
   const int64_t num_blocks = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   if (num_blocks > INT32_MAX) return HDQT_ERR_UNSUPPORTED;
-  const dim3 grid((unsigned)num_blocks);
+  const int sms = sm_count();
+  const dim3 grid((unsigned)(num_blocks < sms ? num_blocks : sms));   // persistent: one CTA per SM
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (tiles_out) {
     return acc_shift ? launch_variant<false, true, true>(ma, mb, p, grid, s)
