@@ -355,3 +355,27 @@ def test_tall_skinny_conv_like_shapes(hdqt):
         assert np.array_equal(ws.codes_a().cpu().numpy(), want["Aq"]), kind
         assert np.array_equal(ws.codes_b().cpu().numpy(), want["Bq"]), kind
         _assert_close(out.cpu().numpy(), want["out"])
+
+
+def test_persistent_ctas_mix_merged_and_clamped_blocks(hdqt):
+    """More output blocks than SMs, with certified, partly certified and uncertifiable blocks interleaved, so
+    that one persistent CTA walks through blocks of different kinds (accumulator hand-over state carries over)."""
+    rng = np.random.default_rng(77)
+    M, N, K = 128 * 21, 256 * 9 + 40, 1024            # 22 x 10 = 220 blocks (incl. ragged edges) on 148 SMs
+    Aq = _sparse_codes(rng, M, K, 0.03)
+    Bq = _sparse_codes(rng, N, K, 0.03)
+    for rb in range(0, M // 128, 3):                   # every third row block: dense codes -> nothing certifies
+        Aq[rb * 128:(rb + 1) * 128] = rng.integers(-8, 8, size=(128, K))
+    for rb in range(1, M // 128, 3):                   # next: one dense stripe of K tiles -> a few clamp tiles
+        Aq[rb * 128:(rb + 1) * 128, 96:160] = rng.integers(-8, 8, size=(128, 64))
+    Bq[:, 96:160] = rng.integers(-8, 8, size=(N, 64))
+    want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 0.25, 0.5)
+    na, nb = _dev(_tile_norms(Aq)), _dev(_tile_norms(Bq))
+    qa, qb = torch.tensor([0.25], device="cuda"), torch.tensor([0.5], device="cuda")
+    status = hdqt.new_status("cuda")
+    for flags in (0, hdqt.FLAG_NO_MERGE):
+        out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), qa, qb, want_S=True, norms_a=na, norms_b=nb, flags=flags,
+                                       dev_status=status)
+        hdqt.check_device_status(status)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), flags
+        assert np.array_equal(out.cpu().numpy(), want_out), flags
