@@ -99,14 +99,14 @@ def test_host_side_rejections(hdqt):
     assert q(256, 4, 32, 32, 1, 32, 4, 1.0, 0, 0, 0, None, 256, 256, None, 256, 8, None, None) == WS
     # integer GEMM argument checks
     g = lib.hdqt_gemm_i8_tiled
-    assert g(256, 256, 256, 256, 8, 8, 48, 4, 8, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 256, None, None) == INVALID
-    assert g(256, 256, 256, 256, 8, 8, 64, 4, 40, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 256, None, None) == INVALID
-    assert g(256, 256, 256, 256, 8, 8, 64, 4, 8, 48, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 256, None, None) == INVALID
-    assert g(256, 256, 256, 256, 8, 8, 64, 4, 8, 32, 0, 32, 256, 4, None, None, 0, None, None, 0, 256, 256, None, None) == INVALID
-    assert g(264, 256, 256, 256, 8, 8, 64, 4, 8, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 256, None, None) == ALIGN
+    assert g(256, 256, 256, 256, 8, 8, 48, 4, 8, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 4096, None, None) == INVALID
+    assert g(256, 256, 256, 256, 8, 8, 64, 4, 40, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 4096, None, None) == INVALID
+    assert g(256, 256, 256, 256, 8, 8, 64, 4, 8, 48, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 4096, None, None) == INVALID
+    assert g(256, 256, 256, 256, 8, 8, 64, 4, 8, 32, 0, 32, 256, 4, None, None, 0, None, None, 0, 256, 4096, None, None) == INVALID
+    assert g(264, 256, 256, 256, 8, 8, 64, 4, 8, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 4096, None, None) == ALIGN
     # per-tile debug output in int8 cannot hold 12-bit accumulators
-    assert g(256, 256, 256, 256, 8, 8, 64, 4, 12, 32, 0, 32, 256, 8, None, 256, 1, None, None, 0, 256, 256, None, None) == INVALID
+    assert g(256, 256, 256, 256, 8, 8, 64, 4, 12, 32, 0, 32, 256, 8, None, 256, 1, None, None, 0, 256, 4096, None, None) == INVALID
     # code_bits outside 2..8
-    assert g(256, 256, 256, 256, 8, 8, 64, 9, 8, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 256, None, None) == INVALID
+    assert g(256, 256, 256, 256, 8, 8, 64, 9, 8, 32, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 4096, None, None) == INVALID
     # a wide sum that could overflow int32 is refused
-    assert g(256, 256, 256, 256, 8, 8, 1 << 22, 8, 32, 0, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 256, None, None) == UNSUPPORTED
+    assert g(256, 256, 256, 256, 8, 8, 1 << 22, 8, 32, 0, 0, 32, 256, 8, None, None, 0, None, None, 0, 256, 4096, None, None) == UNSUPPORTED
