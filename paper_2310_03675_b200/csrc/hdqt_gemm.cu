@@ -345,18 +345,19 @@ __device__ __forceinline__ float dequant_scale(const GemmParams& p) {
 // Staged path: the warp's 32 x 16 block is transposed through a 2 KB shared-memory box so that every
 // store instruction writes 8 rows x 64 contiguous bytes (whole sectors) instead of 32 rows x 16 bytes;
 // stores are fire-and-forget, so the box can be reused as soon as the warp has read it back.
+// raw = true parks the integer sums themselves (as bit patterns) for a later fix-up pass instead.
 __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e, const BlockJob& job, int c,
-                                            int (&val)[16], bool parked, float scale) {
+                                            int (&val)[16], bool parked, float scale, bool raw = false) {
   const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
   const int64_t gn = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16;
   const bool staged = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
                       (gn + 16 <= p.N);    // warp-uniform
   if (staged) {
-    if (gm < p.M && (parked || p.S_out != nullptr)) {
+    if (gm < p.M && (parked || (p.S_out != nullptr && !raw))) {
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         if (parked) val[i] += __float_as_int(p.out[gm * p.ld_out + gn + i]);
-        if (p.S_out != nullptr) p.S_out[gm * p.N + gn + i] = val[i];
+        if (p.S_out != nullptr && !raw) p.S_out[gm * p.N + gn + i] = val[i];
       }
     }
     // row r of the box starts at r*16 floats; the four float4 of a row are rotated by (r >> 1) & 3 so
@@ -365,8 +366,11 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
     const int rot = (e.lane >> 1) & 3;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      dst[(i + rot) & 3] = make_float4(__fmul_rn((float)val[4 * i], scale), __fmul_rn((float)val[4 * i + 1], scale),
-                                       __fmul_rn((float)val[4 * i + 2], scale), __fmul_rn((float)val[4 * i + 3], scale));
+      dst[(i + rot) & 3] =
+          raw ? make_float4(__int_as_float(val[4 * i]), __int_as_float(val[4 * i + 1]), __int_as_float(val[4 * i + 2]),
+                            __int_as_float(val[4 * i + 3]))
+              : make_float4(__fmul_rn((float)val[4 * i], scale), __fmul_rn((float)val[4 * i + 1], scale),
+                            __fmul_rn((float)val[4 * i + 2], scale), __fmul_rn((float)val[4 * i + 3], scale));
     }
     __syncwarp();
     const int sub = e.lane >> 2, quad = e.lane & 3;       // 8 rows per instruction, 4 lanes per row
@@ -382,7 +386,8 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
 #pragma unroll
     for (int i = 0; i < 16; i += 4) {
       int s4[4] = {val[i], val[i + 1], val[i + 2], val[i + 3]};
-      emit4<true>(p, gm, gn + i, s4, parked, false, scale);
+      if (raw) emit4<false>(p, gm, gn + i, s4, parked, false, scale);
+      else emit4<true>(p, gm, gn + i, s4, parked, false, scale);
     }
   }
 }
@@ -916,10 +921,27 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
 constexpr int PAIR_M = 2 * BM;
 
-// flag[t] = 1 iff pair block t (grouped order over [tiles_m2, tiles_n]) is clamp-free for every 32-wide K tile
+// Class of pair block t (grouped order over [tiles_m2, tiles_n]) from the number u of its accumulator tiles
+// without a clamp-free certificate:  1 = none (pure),  2 = a few (u <= max_fix: the pair kernel accumulates them
+// unclamped and a fix-up pass repairs the sums),  0 = many (general kernel).
+constexpr int kFixFlag = 0x40000000;   // marks class-2 blocks in the pair kernel's work list
+
+__device__ __forceinline__ bool pair_tile_certified(const int32_t* a0, const int32_t* b0, int64_t T, bool has_a1,
+                                                    bool has_b1, int t0, int t1, int64_t thr_sq) {
+  bool ok = true;
+  for (int k = t0; k < t1; ++k) {
+    int64_t a2 = __ldg(a0 + k), b2 = __ldg(b0 + k);
+    if (has_a1) a2 = max(a2, (int64_t)__ldg(a0 + T + k));
+    if (has_b1) b2 = max(b2, (int64_t)__ldg(b0 + T + k));
+    ok = ok && (a2 * b2 <= thr_sq);
+  }
+  return ok;
+}
+
 __global__ void classify_pair_blocks_kernel(const int32_t* __restrict__ norms_a, const int32_t* __restrict__ norms_b,
-                                            int64_t M, int64_t N, int tiles32, int64_t thr_sq, int tiles_m2,
-                                            int tiles_n, uint8_t* __restrict__ flag) {
+                                            int64_t M, int64_t N, int tiles32, int tiles_per_acc, int num_acc,
+                                            int64_t thr_sq, int max_fix, int tiles_m2, int tiles_n,
+                                            uint8_t* __restrict__ flag) {
   const int warps_per_block = blockDim.x >> 5;
   const int t = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -931,34 +953,34 @@ __global__ void classify_pair_blocks_kernel(const int32_t* __restrict__ norms_a,
   const int32_t* b0 = norms_b + (int64_t)(2 * tn) * T;
   const bool has_a1 = (int64_t)(2 * tm + 1) * 128 < M;
   const bool has_b1 = (int64_t)(2 * tn + 1) * 128 < N;
-  bool ok = true;
-  for (int k = lane; k < tiles32; k += 32) {
-    int64_t a2 = __ldg(a0 + k), b2 = __ldg(b0 + k);
-    if (has_a1) a2 = max(a2, (int64_t)__ldg(a0 + T + k));
-    if (has_b1) b2 = max(b2, (int64_t)__ldg(b0 + T + k));
-    ok = ok && (a2 * b2 <= thr_sq);
+  int u = 0;
+  for (int a = lane; a < num_acc; a += 32) {
+    const int t0 = a * tiles_per_acc, t1 = min(tiles32, t0 + tiles_per_acc);
+    u += pair_tile_certified(a0, b0, T, has_a1, has_b1, t0, t1, thr_sq) ? 0 : 1;
   }
-  ok = __all_sync(0xFFFFFFFFu, ok);
-  if (lane == 0) flag[t] = ok ? 1 : 0;
+  u = __reduce_add_sync(0xFFFFFFFFu, u);
+  if (lane == 0) flag[t] = (u == 0) ? 1 : (u <= max_fix ? 2 : 0);
 }
 
 // One thread block: ordered compaction of the flags into the list of clamp-free pair blocks and the list of
 // 128 x 256 blocks (ids = row block * tiles_n + column block) that the general kernel has to do.
 __global__ void __launch_bounds__(1024)
 compact_blocks_kernel(const uint8_t* __restrict__ flag, int tiles_m2, int tiles_n, int64_t M,
-                      int32_t* __restrict__ list_pair, int32_t* __restrict__ list_single, int32_t* __restrict__ counts) {
+                      int32_t* __restrict__ list_pair, int32_t* __restrict__ list_single,
+                      int32_t* __restrict__ list_fix, int32_t* __restrict__ counts) {
   __shared__ int s_warp_pair[32], s_warp_single[32];
-  __shared__ int s_base_pair, s_base_single;
+  __shared__ int s_base_pair, s_base_single, s_fix;
   const int n = tiles_m2 * tiles_n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) { s_base_pair = 0; s_base_single = 0; }
+  if (threadIdx.x == 0) { s_base_pair = 0; s_base_single = 0; s_fix = 0; }
   __syncthreads();
   for (int base = 0; base < n; base += 1024) {
     const int t = base + threadIdx.x;
-    int tm = 0, tn = 0, is_pair = 0, singles = 0;
+    int tm = 0, tn = 0, is_pair = 0, singles = 0, cls = 0;
     if (t < n) {
       tile_coords(t, tiles_m2, tiles_n, tm, tn);
-      is_pair = flag[t];
+      cls = flag[t];
+      is_pair = (cls != 0);
       if (!is_pair) singles = ((int64_t)(2 * tm + 1) * 128 < M) ? 2 : 1;
     }
     // exclusive scans inside the warp
@@ -983,14 +1005,15 @@ compact_blocks_kernel(const uint8_t* __restrict__ flag, int tiles_m2, int tiles_
     __syncthreads();
     const int off_pair = s_base_pair + (warp ? s_warp_pair[warp - 1] : 0) + sp - is_pair;
     const int off_single = s_base_single + (warp ? s_warp_single[warp - 1] : 0) + ss - singles;
-    if (is_pair) list_pair[off_pair] = t;
+    if (is_pair) list_pair[off_pair] = t | (cls == 2 ? kFixFlag : 0);
+    if (cls == 2) list_fix[atomicAdd(&s_fix, 1)] = t;      // order is irrelevant for the fix-up pass
     if (singles >= 1) list_single[off_single] = (2 * tm) * tiles_n + tn;
     if (singles == 2) list_single[off_single + 1] = (2 * tm + 1) * tiles_n + tn;
     __syncthreads();
     if (threadIdx.x == 0) { s_base_pair += s_warp_pair[31]; s_base_single += s_warp_single[31]; }
     __syncthreads();
   }
-  if (threadIdx.x == 0) { counts[0] = s_base_pair; counts[1] = s_base_single; }
+  if (threadIdx.x == 0) { counts[0] = s_base_pair; counts[1] = s_base_single; counts[2] = s_fix; }
 }
 
 // ---- cta_group::2 kernel for clamp-free pair blocks ---------------------------------------------------
@@ -1103,9 +1126,11 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // i-th block of this launch; returns true if its sums are to be parked as integers for the fix-up pass
   auto block_at = [&](int i, int& tm, int& tn) {
     const int t = (p.block_list != nullptr) ? __ldg(p.block_list + i) : i;
-    tile_coords(t, tiles_m2, tiles_n, tm, tn);
+    tile_coords(t & ~kFixFlag, tiles_m2, tiles_n, tm, tn);
+    return (t & kFixFlag) != 0;
   };
 
   if (warp == 0) {
@@ -1181,7 +1206,7 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     for (int i = pair_id; i < num_blocks; i += num_pairs, ++bi) {
       const int buf = bi & 1;
       int tm, tn;
-      block_at(i, tm, tn);
+      const bool raw = block_at(i, tm, tn);
       BlockJob job;
       job.m0 = tm * PAIR_M + (int)cta_rank * BM;
       job.n0 = tn * BN;
@@ -1204,7 +1229,7 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         int val[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) val[k] = (int)mv[c * 16 + k];
-        store_chunk(p, e, job, c, val, false, scale);
+        store_chunk(p, e, job, c, val, false, scale, raw);
       }
     }
   }
@@ -1218,6 +1243,132 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
                  : "memory");
   }
   if (threadIdx.x == 0 && *abort_flag) report_status(p.dev_status, HDQT_ERR_TIMEOUT);
+}
+
+// ---- fix-up pass for pair blocks with a few uncertified accumulator tiles -----------------------------
+// The pair kernel accumulated ALL their tiles unclamped and parked the integer sums in the output buffer.
+// For an uncertified tile the accumulator quantisation may change the tile sum, so this pass recomputes
+// exactly those tile sums P on the CUDA cores and adds clamp(P) - P; the result is sum_t clamp(P_t) bit for bit
+// (on certified tiles the clamp is the identity).  Then it applies the dequantising scale.
+// Work item = one 128-row half of a 256 x 256 block, 512 threads: warp w owns rows 8w..8w+7, lane l owns the
+// columns l + 32 j.  Corrections are rare, so they are added to the parked sums in place as they are found.
+constexpr int kMaxFixTiles = 256;   // the classification sends blocks with more uncertified tiles to the general kernel
+constexpr int FIX_B_STRIDE = 36;    // bytes per staged B row (32 + 4: consecutive rows fall into different banks)
+
+__global__ void __launch_bounds__(512)
+fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict__ Bq, const GemmParams p,
+                         const int32_t* __restrict__ list_fix, const int32_t* __restrict__ counts) {
+  __shared__ __align__(16) uint8_t sA[128 * 32];
+  __shared__ __align__(16) uint8_t sB[256 * FIX_B_STRIDE];
+  __shared__ int s_list[kMaxFixTiles];
+  __shared__ int s_count;
+  const int tiles_m2 = (int)((p.M + PAIR_M - 1) / PAIR_M), tiles_n = (int)((p.N + BN - 1) / BN);
+  const int n_items = 2 * __ldg(counts + 2);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t T = p.tiles32;
+  const float scale = dequant_scale(p);
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    int tm, tn;
+    tile_coords(__ldg(list_fix + (item >> 1)), tiles_m2, tiles_n, tm, tn);
+    const int64_t m0 = (int64_t)tm * PAIR_M + (item & 1) * BM, n0 = (int64_t)tn * BN;
+    if (m0 >= p.M) continue;     // block-uniform: the lower half of a ragged last block does not exist
+    // certificates are those of the whole pair block (what the pair kernel relied on)
+    const int32_t* a0 = p.norms_a + (int64_t)(2 * tm) * T;
+    const int32_t* b0 = p.norms_b + (int64_t)(2 * tn) * T;
+    const bool has_a1 = (int64_t)(2 * tm + 1) * 128 < p.M;
+    const bool has_b1 = (int64_t)(2 * tn + 1) * 128 < p.N;
+    // all threads look for the (few) uncertified accumulator tiles in parallel, then walk that short list
+    __syncthreads();
+    if (threadIdx.x == 0) s_count = 0;
+    __syncthreads();
+    for (int a = threadIdx.x; a < p.num_acc; a += blockDim.x) {
+      const int t0 = a * p.tiles_per_acc, t1 = min(p.tiles32, t0 + p.tiles_per_acc);
+      if (!pair_tile_certified(a0, b0, T, has_a1, has_b1, t0, t1, p.cert_thr_sq)) {
+        const int slot = atomicAdd(&s_count, 1);
+        if (slot < kMaxFixTiles) s_list[slot] = a;
+      }
+    }
+    __syncthreads();
+    const int n_uncert = min(s_count, kMaxFixTiles);
+    for (int u = 0; u < n_uncert; ++u) {
+      const int a = s_list[u];
+      const int t0 = a * p.tiles_per_acc, t1 = min(p.tiles32, t0 + p.tiles_per_acc);
+      int P[8][8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) P[r][j] = 0;
+      for (int t = t0; t < t1; ++t) {
+        __syncthreads();
+        {   // stage the 32-byte K slice of 128 rows of A and 256 rows of B (rows beyond the matrices read as zero)
+          const int row = threadIdx.x >> 2, part = threadIdx.x & 3;     // 4 threads x 8 bytes per row
+          uint2 va = make_uint2(0u, 0u);
+          if (m0 + row < p.M) va = __ldg(reinterpret_cast<const uint2*>(Aq + (m0 + row) * p.K_pad + (int64_t)t * 32 + part * 8));
+          *reinterpret_cast<uint2*>(sA + row * 32 + part * 8) = va;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int brow = row + 128 * h;
+            uint2 vb = make_uint2(0u, 0u);
+            if (n0 + brow < p.N) vb = __ldg(reinterpret_cast<const uint2*>(Bq + (n0 + brow) * p.K_pad + (int64_t)t * 32 + part * 8));
+            uint32_t* db = reinterpret_cast<uint32_t*>(sB + brow * FIX_B_STRIDE + part * 8);
+            db[0] = vb.x;
+            db[1] = vb.y;
+          }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          int av[8], bv[8];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) av[r] = *reinterpret_cast<const int*>(sA + (warp * 8 + r) * 32 + k * 4);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) bv[j] = *reinterpret_cast<const int*>(sB + (lane + 32 * j) * FIX_B_STRIDE + k * 4);
+#pragma unroll
+          for (int r = 0; r < 8; ++r)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) P[r][j] = __dp4a(av[r], bv[j], P[r][j]);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        const int64_t gm = m0 + warp * 8 + r;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int64_t gn = n0 + lane + 32 * j;
+          const int d = min(max(P[r][j], p.lo), p.hi) - P[r][j];
+          if (d != 0 && gm < p.M && gn < p.N) {
+            int* o = reinterpret_cast<int*>(p.out + gm * p.ld_out + gn);   // only this thread touches this element
+            *o += d;
+          }
+        }
+      }
+    }
+    // parked (now exact) integer sums -> fp32, lanes on consecutive columns; all loads first, so that
+    // they are in flight together (each element is touched by this thread only)
+    int Sv[8][8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const int64_t gm = m0 + warp * 8 + r;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int64_t gn = n0 + lane + 32 * j;
+        Sv[r][j] = (gm < p.M && gn < p.N) ? __float_as_int(__ldcg(p.out + gm * p.ld_out + gn)) : 0;
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const int64_t gm = m0 + warp * 8 + r;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int64_t gn = n0 + lane + 32 * j;
+        if (gm < p.M && gn < p.N) {
+          p.out[gm * p.ld_out + gn] = __fmul_rn((float)Sv[r][j], scale);
+          if (p.S_out != nullptr) p.S_out[gm * p.N + gn] = Sv[r][j];
+        }
+      }
+    }
+    __syncthreads();
+  }
 }
 
 // ---- smallest clamp-free accumulator shift (CUDA cores; a calibration utility, not the hot path)
@@ -1300,9 +1451,9 @@ using namespace hdqt;
 
 namespace {
 inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
-// scratch of the work split: [counts 256 B | flags u8[npb] | pair list i32[npb] | single list i32[2 npb]]
+// scratch of the work split: [counts 256 B | classes u8[npb] | pair list i32[npb] | single list i32[2 npb] | fix list i32[npb]]
 struct SplitLayout {
-  size_t flags, list_pair, list_single, total;
+  size_t flags, list_pair, list_single, list_fix, total;
   int64_t npb;
 };
 inline SplitLayout split_layout(int64_t M, int64_t N) {
@@ -1311,7 +1462,8 @@ inline SplitLayout split_layout(int64_t M, int64_t N) {
   L.flags = 256;
   L.list_pair = L.flags + up256((size_t)L.npb);
   L.list_single = L.list_pair + up256((size_t)L.npb * 4);
-  L.total = L.list_single + up256((size_t)L.npb * 8);
+  L.list_fix = L.list_single + up256((size_t)L.npb * 8);
+  L.total = L.list_fix + up256((size_t)L.npb * 4);
   return L;
 }
 }  // namespace
@@ -1401,9 +1553,10 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
   dim3 grid((unsigned)(num_blocks < sms ? num_blocks : sms));   // persistent: one CTA per SM
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 
-  // Large problems with clamp-free tiles: split the output blocks between the cta_group::2 kernel (blocks
-  // whose every K tile is certified) and the general kernel (the rest).
-  const bool split = (p.merge != 0) && !tiles_out && num_blocks >= 2 * (int64_t)sms && sms >= 2 && workspace != nullptr;
+  // Large problems (at least 8 output blocks per SM; below that the extra launches cost more than they gain)
+  // with clamp-free tiles: the cta_group::2 kernel takes the blocks whose K tiles are all, or all but a few,
+  // certified (a fix-up pass repairs the few), the general kernel takes the rest.
+  const bool split = (p.merge != 0) && !tiles_out && num_blocks >= 8 * (int64_t)sms && sms >= 2 && workspace != nullptr;
   if (split) {
     const SplitLayout L = split_layout(M, N);
     if (L.npb > INT32_MAX / 4) return HDQT_ERR_UNSUPPORTED;
@@ -1416,10 +1569,14 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
     CUtensorMap mb_half;
     if (!make_operand_map(&mb_half, Bq, N, K_pad, BN / 2)) return HDQT_ERR_CUDA;
     GemmParams pp = p;
+    int32_t* list_fix = reinterpret_cast<int32_t*>(ws + L.list_fix);
     if (p.merge == 1) {
-      classify_pair_blocks_kernel<<<(unsigned)((L.npb + 7) / 8), 256, 0, s>>>(norms_a, norms_b, M, N, p.tiles32,
-                                                                             p.cert_thr_sq, tiles_m2, tiles_n, flags);
-      compact_blocks_kernel<<<1, 1024, 0, s>>>(flags, tiles_m2, tiles_n, M, list_pair, list_single, counts);
+      // blocks with at most 1/32 of their accumulator tiles uncertified are repaired by the fix-up pass
+      int max_fix = p.num_acc / 32 > 0 ? p.num_acc / 32 : 1;
+      if (max_fix > kMaxFixTiles) max_fix = kMaxFixTiles;
+      classify_pair_blocks_kernel<<<(unsigned)((L.npb + 7) / 8), 256, 0, s>>>(
+          norms_a, norms_b, M, N, p.tiles32, p.tiles_per_acc, p.num_acc, p.cert_thr_sq, max_fix, tiles_m2, tiles_n, flags);
+      compact_blocks_kernel<<<1, 1024, 0, s>>>(flags, tiles_m2, tiles_n, M, list_pair, list_single, list_fix, counts);
       pp.block_list = list_pair;
       pp.block_count = counts;
     }   // merge == 2: every block is clamp-free whatever the data, no lists needed
@@ -1431,6 +1588,8 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_failure(e, "launch(pair gemm)");
     if (p.merge == 2) return HDQT_OK;
+    fixup_pair_blocks_kernel<<<(unsigned)(2 * sms), 512, 0, s>>>(Aq, Bq, p, list_fix, counts);
+    if (cudaGetLastError() != cudaSuccess) return HDQT_ERR_CUDA;
     p.block_list = list_single;     // the general kernel does what is left
     p.block_count = counts + 1;
   }

@@ -379,3 +379,40 @@ def test_persistent_ctas_mix_merged_and_clamped_blocks(hdqt):
         hdqt.check_device_status(status)
         assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), flags
         assert np.array_equal(out.cpu().numpy(), want_out), flags
+
+
+def test_work_split_pure_fixup_and_general_blocks(hdqt):
+    """Large enough for the work split (>= 8 blocks per SM): pair blocks that are fully certified, that have a
+    few uncertified tiles (fix-up pass) and that have many (general kernel), with ragged edges."""
+    rng = np.random.default_rng(88)
+    M, N, K = 128 * 37 + 50, 256 * 33 + 24, 2048            # 38 x 34 = 1292 single blocks >= 8 x 148
+    Aq = (rng.integers(-1, 2, size=(M, K)) * (rng.random((M, K)) < 0.05)).astype(np.int8)   # tiny norms: certifiable
+    Bq = (rng.integers(-1, 2, size=(N, K)) * (rng.random((N, K)) < 0.05)).astype(np.int8)
+    for rb in range(0, M // 128, 5):                         # dense row blocks: nothing certifies there
+        Aq[rb * 128:(rb + 1) * 128] = rng.integers(-8, 8, size=(128, K))
+    Bq[:, ::3] = np.where(Bq[:, ::3] == 0, 3, Bq[:, ::3])    # enough weight in B for the dense A blocks to fail
+    for rb in range(2, M // 128, 5):                         # one dense 32-wide K tile: a single uncertified tile
+        Aq[rb * 128:(rb + 1) * 128, 320:352] = rng.integers(-8, 8, size=(128, 32))
+    Bq[:, 320:352] = rng.integers(-8, 8, size=(N, 32))
+    Bq[:, 1024:1056] = rng.integers(6, 8, size=(N, 32))      # large codes: these tiles really clamp
+    Aq[2 * 128:3 * 128, 1024:1056] = rng.integers(6, 8, size=(128, 32))
+    want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 0.25, 0.5)
+    na, nb = _dev(_tile_norms(Aq)), _dev(_tile_norms(Bq))
+    qa, qb = torch.tensor([0.25], device="cuda"), torch.tensor([0.5], device="cuda")
+    status = hdqt.new_status("cuda")
+    out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), qa, qb, want_S=True, norms_a=na, norms_b=nb, dev_status=status)
+    hdqt.check_device_status(status)
+    assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
+    assert np.array_equal(out.cpu().numpy(), want_out)
+    # the classes really occur: a fully certified pair block, one with a few uncertified tiles, one with many
+    na64, nb64 = _tile_norms(Aq).astype(np.int64), _tile_norms(Bq).astype(np.int64)
+    def uncert(tm, tn):
+        a = na64[2 * tm:2 * tm + 2].max(0)
+        b = nb64[2 * tn:2 * tn + 2].max(0)
+        return int((a * b > 127 * 127).sum())
+    counts = sorted({min(uncert(tm, 0), 3) for tm in range(M // 256)})
+    assert counts[0] == 0 and 1 in counts + [2] and counts[-1] == 3
+    # wide accumulators: every block goes to the pair kernel without certificates
+    out16, S16, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), qa, qb, acc_bits=16, want_S=True, dev_status=status)
+    hdqt.check_device_status(status)
+    assert np.array_equal(S16.cpu().numpy().astype(np.int64), Aq.astype(np.int64) @ Bq.astype(np.int64).T)
