@@ -28,9 +28,9 @@ sys.path.insert(0, ROOT)
 METRIC = "hdqt_gemm_int_tops"
 UNIT = "TOPS"
 SEED = 1234
-# dram__bytes_read.sum + dram__bytes_write.sum of one gemm_i8_tiled_kernel launch at M=N=K=8192 (merged path),
+# dram__bytes_read.sum + dram__bytes_write.sum of the GEMM kernels of one step at M=N=K=8192 (pair kernel + fix-up),
 # from the ncu capture summarised in profiles/gemm_i8_tiled_kernel_sweep.md
-GEMM_DRAM_BYTES_8192 = 360.1e6 + 243.3e6
+GEMM_DRAM_BYTES_8192 = 301.8e6 + 241.0e6 + 36.5e6 + 0.3e6
 
 
 def parse_args():
@@ -182,6 +182,20 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
+
+def launches_per_step(M, N, merge, wgrad, acc_bits, sms=148):
+    """Kernels of this library launched by one step (what the host layer does, restated for the report):
+    2 calibration + 2 quantize kernels, the tile-norm reduction for K-contiguous operands when merging, and the
+    GEMM: one kernel, or - at >= 8 output blocks per SM with merging - classify, compact, pair kernel, fix-up and
+    general kernel (the pair kernel alone when the accumulators are too wide to clamp)."""
+    n = 4 + (2 if (merge and not wgrad) else 0)
+    blocks = ((M + 127) // 128) * ((N + 255) // 256)
+    if merge and blocks >= 8 * sms:
+        n += 1 if acc_bits >= 13 else 5
+    else:
+        n += 1
+    return n
+
 
 def max_over_ranks(values, device, world):
     """Element-wise maximum of per-rank timings over all ranks (every rank gets the result)."""
@@ -352,7 +366,7 @@ def run_hdqt(args):
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f32",
             "data": "synthetic", "config": workload_config(size, merge, args.layout, args.acc_tile, args.acc_bits),
-            "roofline": {"bound": "tensor", "kernel": "gemm_i8_tiled_kernel", "achieved": gemm_tops,
+            "roofline": {"bound": "tensor", "kernel": "hdqt_gemm_i8_tiled (pair kernel + fix-up + general kernel)", "achieved": gemm_tops,
                          "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak, "peak_source": peak_src,
                          "traffic": GEMM_DRAM_BYTES_8192 if (size == 8192 and merge and not wgrad) else None,
                          "traffic_unit": "bytes per launch (ncu dram read+write, profiles/gemm_i8_tiled_kernel_sweep.md)",
@@ -362,7 +376,7 @@ def run_hdqt(args):
                          "gbs": quant_bytes / (quant_ms * 1e-3) / 1e9, "hbm_peak_gbs": hbm,
                          "frac": quant_bytes / (quant_ms * 1e-3) / 1e9 / hbm,
                          "note": "both operands: calibration pass (4 B/elt) + FWHT/quantize pass (5 B/elt)"},
-            "clocks": clocks, "gpu_launches": args.steps * (5 + (2 if (merge and not wgrad) else 0)),
+            "clocks": clocks, "gpu_launches": args.steps * launches_per_step(M, N, merge, wgrad, desc.acc_bits),
         }
         if e2e is not None:
             line["e2e"] = e2e
