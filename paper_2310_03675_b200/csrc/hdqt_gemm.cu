@@ -1250,28 +1250,30 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 // For an uncertified tile the accumulator quantisation may change the tile sum, so this pass recomputes
 // exactly those tile sums P on the CUDA cores and adds clamp(P) - P; the result is sum_t clamp(P_t) bit for bit
 // (on certified tiles the clamp is the identity).  Then it applies the dequantising scale.
-// Work item = one 128-row half of a 256 x 256 block, 512 threads: warp w owns rows 8w..8w+7, lane l owns the
-// columns l + 32 j.  Corrections are rare, so they are added to the parked sums in place as they are found.
+// Work item = 64 rows of a 256 x 256 block (4 items per block, so that the few blocks spread over all SMs),
+// 256 threads: warp w owns rows 8w..8w+7, lane l owns the columns l + 32 j.  Corrections are rare, so they are
+// added to the parked sums in place as they are found.
+constexpr int FIX_ROWS = 64;
 constexpr int kMaxFixTiles = 256;   // the classification sends blocks with more uncertified tiles to the general kernel
 constexpr int FIX_B_STRIDE = 36;    // bytes per staged B row (32 + 4: consecutive rows fall into different banks)
 
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(256, 2)
 fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict__ Bq, const GemmParams p,
                          const int32_t* __restrict__ list_fix, const int32_t* __restrict__ counts) {
-  __shared__ __align__(16) uint8_t sA[128 * 32];
+  __shared__ __align__(16) uint8_t sA[FIX_ROWS * 32];
   __shared__ __align__(16) uint8_t sB[256 * FIX_B_STRIDE];
   __shared__ int s_list[kMaxFixTiles];
   __shared__ int s_count;
   const int tiles_m2 = (int)((p.M + PAIR_M - 1) / PAIR_M), tiles_n = (int)((p.N + BN - 1) / BN);
-  const int n_items = 2 * __ldg(counts + 2);
+  const int n_items = (PAIR_M / FIX_ROWS) * __ldg(counts + 2);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t T = p.tiles32;
   const float scale = dequant_scale(p);
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
     int tm, tn;
-    tile_coords(__ldg(list_fix + (item >> 1)), tiles_m2, tiles_n, tm, tn);
-    const int64_t m0 = (int64_t)tm * PAIR_M + (item & 1) * BM, n0 = (int64_t)tn * BN;
-    if (m0 >= p.M) continue;     // block-uniform: the lower half of a ragged last block does not exist
+    tile_coords(__ldg(list_fix + item / (PAIR_M / FIX_ROWS)), tiles_m2, tiles_n, tm, tn);
+    const int64_t m0 = (int64_t)tm * PAIR_M + (item % (PAIR_M / FIX_ROWS)) * FIX_ROWS, n0 = (int64_t)tn * BN;
+    if (m0 >= p.M) continue;     // block-uniform: these rows of a ragged last block do not exist
     // certificates are those of the whole pair block (what the pair kernel relied on)
     const int32_t* a0 = p.norms_a + (int64_t)(2 * tm) * T;
     const int32_t* b0 = p.norms_b + (int64_t)(2 * tn) * T;
@@ -1300,14 +1302,14 @@ fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict
         for (int j = 0; j < 8; ++j) P[r][j] = 0;
       for (int t = t0; t < t1; ++t) {
         __syncthreads();
-        {   // stage the 32-byte K slice of 128 rows of A and 256 rows of B (rows beyond the matrices read as zero)
+        {   // stage the 32-byte K slice of 64 rows of A and 256 rows of B (rows beyond the matrices read as zero)
           const int row = threadIdx.x >> 2, part = threadIdx.x & 3;     // 4 threads x 8 bytes per row
           uint2 va = make_uint2(0u, 0u);
           if (m0 + row < p.M) va = __ldg(reinterpret_cast<const uint2*>(Aq + (m0 + row) * p.K_pad + (int64_t)t * 32 + part * 8));
           *reinterpret_cast<uint2*>(sA + row * 32 + part * 8) = va;
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int brow = row + 128 * h;
+          for (int h = 0; h < 256 / FIX_ROWS; ++h) {
+            const int brow = row + FIX_ROWS * h;
             uint2 vb = make_uint2(0u, 0u);
             if (n0 + brow < p.N) vb = __ldg(reinterpret_cast<const uint2*>(Bq + (n0 + brow) * p.K_pad + (int64_t)t * 32 + part * 8));
             uint32_t* db = reinterpret_cast<uint32_t*>(sB + brow * FIX_B_STRIDE + part * 8);
@@ -1588,7 +1590,7 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_failure(e, "launch(pair gemm)");
     if (p.merge == 2) return HDQT_OK;
-    fixup_pair_blocks_kernel<<<(unsigned)(2 * sms), 512, 0, s>>>(Aq, Bq, p, list_fix, counts);
+    fixup_pair_blocks_kernel<<<(unsigned)(2 * sms), 256, 0, s>>>(Aq, Bq, p, list_fix, counts);
     if (cudaGetLastError() != cudaSuccess) return HDQT_ERR_CUDA;
     p.block_list = list_single;     // the general kernel does what is left
     p.block_count = counts + 1;
