@@ -1,0 +1,553 @@
+// Device-side building blocks of the tiled integer GEMM kernels: tile constants, kernel parameters, PTX
+// wrappers (mbarrier, TMA, tcgen05), and the epilogue of one output block (accumulator quantisation, packed
+// 16-bit-lane sums, staged stores).  Included by hdqt_gemm.cu only (one translation unit).
+#pragma once
+
+#include <cuda.h>
+
+#include "hdqt_common.cuh"
+
+namespace hdqt {
+
+namespace {
+
+
+constexpr int BM = 128;          // output rows per CTA (= TMEM lanes)
+constexpr int BN = 256;          // output columns per CTA (= one MMA's N)
+constexpr int BKB = 128;         // bytes of K per stage row (one 128B swizzle atom = 4 tiles of 32)
+constexpr int STAGES = 4;
+constexpr int A_STAGE = BM * BKB;              // 16 KB
+constexpr int B_STAGE = BN * BKB;              // 32 KB
+constexpr int STAGE_BYTES = A_STAGE + B_STAGE; // 48 KB
+constexpr int NUM_EPI_WARPS = 8;               // 2 per TMEM lane quarter, 128 accumulator columns each
+constexpr int EPI_COLS = BN / (NUM_EPI_WARPS / 4);
+constexpr int GEMM_THREADS = 32 * (3 + NUM_EPI_WARPS);   // + TMA producer, MMA issuer, certificate builder
+constexpr int TMEM_COLS = 512;
+constexpr int MAX_CERT_WORDS = 256;            // certificate bitmask: up to 8192 accumulator tiles
+constexpr int OUT_STAGE_WARP = 32 * 16 * 4;    // per epilogue warp: a 32-row x 16-column fp32 box for the store transpose
+constexpr int TILE_INFO_BYTES = 4 * MAX_CERT_WORDS + 16;
+// the dynamic shared-memory window is declared 1024-byte aligned (checked in the kernel), so no slack is kept
+// offset of the store boxes (128-byte aligned)
+constexpr int OUT_STAGE_OFF = (STAGES * STAGE_BYTES + 256 /*barriers*/ + 2 * TILE_INFO_BYTES + 127) / 128 * 128;
+constexpr int SMEM_BYTES = OUT_STAGE_OFF + NUM_EPI_WARPS * OUT_STAGE_WARP;
+static_assert(OUT_STAGE_WARP % 128 == 0, "store boxes must stay 128-byte aligned");
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+
+// instruction descriptor: D = s32, A = B = signed 8-bit, both K-major, N = 256, M = 128
+constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                           ((uint32_t)(BM >> 4) << 24);
+
+struct GemmParams {
+  int64_t M, N, K_pad;
+  int32_t tiles32;        // K_pad / 32
+  int32_t tiles_per_acc;  // acc_tile / 32 (tiles32 if acc_tile == 0)
+  int32_t num_acc;        // accumulator tiles along K
+  int32_t acc_shift;
+  int32_t lo, hi;         // accumulator range
+  int32_t had_block;
+  int32_t flush_every;    // packed mode: accumulator tiles summed in 16-bit lanes before widening
+  // merging of provably clamp-free accumulator tiles
+  int32_t merge;          // 0 = off, 1 = certificates from the tile norms, 2 = every tile is clamp-free
+  int32_t merge_max_uncert_256;  // a CTA merges only if uncertified tiles <= this/256 of all tiles
+  int64_t cert_thr_sq;    // a 32-wide sub-tile is certified iff norm_a*norm_b <= this
+  const int32_t* norms_a; // [ceil(M/128), tiles32]
+  const int32_t* norms_b; // [ceil(N/128), tiles32]
+  const float* step_a;
+  const float* step_b;
+  float* out;
+  int64_t ld_out;
+  int32_t* S_out;
+  void* tiles_out;
+  int32_t tiles_elem_bytes;
+  int32_t* dev_status;
+  // optional work list (device): when set, the kernel processes block_count[0] output blocks whose ids
+  // (row block * column blocks + column block) are in block_list, instead of all blocks
+  const int32_t* block_list;
+  const int32_t* block_count;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded waits: each gives up after ~1 s, or as soon as another role has given up.
+//
+// mbar_wait: for the two single-thread roles (TMA producer, MMA issuer), whose waits are on the
+// critical path of every K tile: polls without suspending first, then backs off.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < (1 << 12); ++i) {
+    if (mbar_test_wait(bar, parity)) return true;
+  }
+  for (int i = 0; i < (1 << 20); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    __nanosleep(512);
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// mbar_wait_yield: for the epilogue warps. A warp that spins steals issue slots from the MMA issuer
+// and from the warps that have work, so these waits suspend in hardware (try_wait) and sleep between
+// polls; kSleepNs is the poll period (short for the per-tile handshake, long for the one wait on the
+// merged accumulator that spans the whole main loop).
+template <int kSleepNs>
+__device__ __forceinline__ bool mbar_wait_yield(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  constexpr int kLimit = (kSleepNs >= 512) ? (1 << 21) : (1 << 24);
+  for (int i = 0; i < kLimit; ++i) {
+    __nanosleep(kSleepNs);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63) == 63 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(IDESC), "r"(accumulate)
+      : "memory");
+}
+
+// K-major operand tile with 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address
+  d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                         // SWIZZLE_128B
+  return d;
+}
+
+#define HDQT_TMEM_LD32(taddr, v)                                                                        \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                         \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                         \
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"         \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),      \
+        "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),      \
+        "=r"(v[29]), "=r"(v[30]), "=r"(v[31])                                                           \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+#define HDQT_TMEM_LD32_PACK16(taddr, v)                                                                 \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x32.pack::16b.b32 "                                               \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                         \
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"         \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),      \
+        "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),      \
+        "=r"(v[29]), "=r"(v[30]), "=r"(v[31])                                                           \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
+#define HDQT_TMEM_LD16_PACK16(taddr, v)                                                                 \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x16.pack::16b.b32 "                                               \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"                  \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15])                                                                                     \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
+// tcgen05.wait::ld tied to the registers of the load it completes, so that the compiler cannot move
+// their first use above the wait
+#define HDQT_TMEM_WAIT16(v)                                                                             \
+  asm volatile("tcgen05.wait::ld.sync.aligned;"                                                         \
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]),    \
+                 "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), \
+                 "+r"(v[14]), "+r"(v[15])                                                               \
+               :                                                                                        \
+               : "memory")
+
+#define HDQT_TMEM_WAIT32(v)                                                                             \
+  asm volatile("tcgen05.wait::ld.sync.aligned;"                                                         \
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]),    \
+                 "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), \
+                 "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]),          \
+                 "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]),          \
+                 "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])           \
+               :                                                                                        \
+               : "memory")
+
+#define HDQT_TMEM_LD16(taddr, v)                                                                        \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "                                                         \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"                  \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15])                                                                                     \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
+// packed (two columns per register) load of half of a warp's columns, and the matching wait
+#define HDQT_LD_HALF_PACK(taddr, v)                                    \
+  do {                                                                 \
+    if constexpr (EPI_COLS / 4 == 32) { HDQT_TMEM_LD32_PACK16(taddr, v); } \
+    else { HDQT_TMEM_LD16_PACK16(taddr, v); }                          \
+  } while (0)
+#define HDQT_WAIT_HALF(v)                                              \
+  do {                                                                 \
+    if constexpr (EPI_COLS / 4 == 32) { HDQT_TMEM_WAIT32(v); }         \
+    else { HDQT_TMEM_WAIT16(v); }                                      \
+  } while (0)
+
+// accumulator quantisation of one exact tile sum
+template <bool kShift>
+__device__ __forceinline__ int acc_quant(int P, int r, int lo, int hi) {
+  if (kShift) {
+    // round-half-even of P / 2^r:  (P + (2^(r-1) - 1) + ((P >> r) & 1)) >> r
+    P = (P + ((1 << (r - 1)) - 1) + ((P >> r) & 1)) >> r;
+  }
+  return min(max(P, lo), hi);
+}
+
+// Writes 4 consecutive output columns of one row: the final fp32 values (and optionally the integer
+// sums), or - for an intermediate widening of the packed sums - the int32 partial sums, which are
+// parked in the output buffer itself until the final pass reads them back.
+template <bool kFinal>
+__device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t gn, int (&s)[4], bool have_prev,
+                                      bool vec, float scale) {
+  float* orow = p.out + gm * p.ld_out + gn;
+  if (vec) {
+    if (have_prev) {
+      const int4 prev = *reinterpret_cast<const int4*>(orow);
+      s[0] += prev.x; s[1] += prev.y; s[2] += prev.z; s[3] += prev.w;
+    }
+    if (kFinal) {
+      float4 o;
+      o.x = __fmul_rn((float)s[0], scale);
+      o.y = __fmul_rn((float)s[1], scale);
+      o.z = __fmul_rn((float)s[2], scale);
+      o.w = __fmul_rn((float)s[3], scale);
+      *reinterpret_cast<float4*>(orow) = o;
+    } else {
+      *reinterpret_cast<int4*>(orow) = make_int4(s[0], s[1], s[2], s[3]);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (gn + i < p.N) {
+        if (have_prev) s[i] += __float_as_int(orow[i]);
+        orow[i] = kFinal ? __fmul_rn((float)s[i], scale) : __int_as_float(s[i]);
+      }
+    }
+  }
+  if (kFinal && p.S_out != nullptr) {
+    int32_t* srow = p.S_out + gm * p.N + gn;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (gn + i < p.N) srow[i] = s[i];
+    }
+  }
+}
+
+// ---- epilogue of one output block, as separate functions ---------------------------------------
+// Each variant keeps its own register-resident state (sums, load buffers); keeping them out of the
+// kernel body lets the compiler allocate registers per variant instead of for their union.
+
+struct EpiCtx {               // constants of one epilogue warp
+  uint32_t lane_addr;         // TMEM address of this warp's lane quarter and column group in accumulator 0
+  uint32_t bar_tfull;         // [2] accumulator ready
+  uint32_t bar_tempty;        // [2] accumulator drained
+  volatile int* abort_flag;
+  float* box;                 // this warp's 32 x 16 fp32 staging box in shared memory
+  int q, grp, lane;
+};
+
+struct BlockJob {             // one output block as seen by the epilogue
+  int m0, n0;
+  int n_clamp_tiles;          // accumulator tiles that arrive one by one for the clamp path
+  int n_merged;               // accumulator tiles merged in accumulator 0
+  int merging;                // clamp tiles use accumulator 1 only (else they alternate 0 / 1)
+};
+
+__device__ __forceinline__ float dequant_scale(const GemmParams& p) {
+  return (float)((double)__ldg(p.step_a) * (double)__ldg(p.step_b) * (double)(1u << p.acc_shift) /
+                 (double)p.had_block);
+}
+
+// Final integer sums of columns [16c, 16c+16) of this thread's row -> fp32 output.
+// Staged path: the warp's 32 x 16 block is transposed through a 2 KB shared-memory box so that every
+// store instruction writes 8 rows x 64 contiguous bytes (whole sectors) instead of 32 rows x 16 bytes;
+// stores are fire-and-forget, so the box can be reused as soon as the warp has read it back.
+// raw = true parks the integer sums themselves (as bit patterns) for a later fix-up pass instead.
+__device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e, const BlockJob& job, int c,
+                                            int (&val)[16], bool parked, float scale, bool raw = false) {
+  const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
+  const int64_t gn = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16;
+  const bool staged = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+                      (gn + 16 <= p.N);    // warp-uniform
+  if (staged) {
+    if (gm < p.M && (parked || (p.S_out != nullptr && !raw))) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        if (parked) val[i] += __float_as_int(p.out[gm * p.ld_out + gn + i]);
+        if (p.S_out != nullptr && !raw) p.S_out[gm * p.N + gn + i] = val[i];
+      }
+    }
+    // row r of the box starts at r*16 floats; the four float4 of a row are rotated by (r >> 1) & 3 so
+    // that neither the row-wise writes nor the read-back hit a shared-memory bank twice
+    float4* dst = reinterpret_cast<float4*>(e.box + e.lane * 16);
+    const int rot = (e.lane >> 1) & 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      dst[(i + rot) & 3] =
+          raw ? make_float4(__int_as_float(val[4 * i]), __int_as_float(val[4 * i + 1]), __int_as_float(val[4 * i + 2]),
+                            __int_as_float(val[4 * i + 3]))
+              : make_float4(__fmul_rn((float)val[4 * i], scale), __fmul_rn((float)val[4 * i + 1], scale),
+                            __fmul_rn((float)val[4 * i + 2], scale), __fmul_rn((float)val[4 * i + 3], scale));
+    }
+    __syncwarp();
+    const int sub = e.lane >> 2, quad = e.lane & 3;       // 8 rows per instruction, 4 lanes per row
+#pragma unroll
+    for (int rr = 0; rr < 32; rr += 8) {
+      const int rloc = rr + sub;
+      const float4 v = *reinterpret_cast<const float4*>(e.box + rloc * 16 + ((quad + ((rloc >> 1) & 3)) & 3) * 4);
+      const int64_t grow = (int64_t)job.m0 + e.q * 32 + rloc;
+      if (grow < p.M) *reinterpret_cast<float4*>(p.out + grow * p.ld_out + gn + quad * 4) = v;
+    }
+    __syncwarp();
+  } else if (gm < p.M) {
+#pragma unroll
+    for (int i = 0; i < 16; i += 4) {
+      int s4[4] = {val[i], val[i + 1], val[i + 2], val[i + 3]};
+      if (raw) emit4<false>(p, gm, gn + i, s4, parked, false, scale);
+      else emit4<true>(p, gm, gn + i, s4, parked, false, scale);
+    }
+  }
+}
+
+__device__ __forceinline__ void release_accumulator(const EpiCtx& e, int buf, uint32_t* drains) {
+  tc_fence_before();
+  __syncwarp();
+  if (e.lane == 0) mbar_arrive(e.bar_tempty + 8 * buf);
+  ++drains[buf];
+}
+
+// Whole block merged (the common case on heavy-tailed operands): no per-tile sums exist, so the registers
+// take the complete accumulator row at once and the accumulator goes back to the MMA issuer before any
+// conversion or store work.
+__device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+  if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+  tc_fence_after();
+  const float scale = dequant_scale(p);
+  uint32_t mv[EPI_COLS];
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) HDQT_TMEM_LD16(e.lane_addr + c * 16, (mv + c * 16));
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) HDQT_TMEM_WAIT16((mv + c * 16));
+  release_accumulator(e, 0, drains);
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) {
+    int val[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) val[i] = (int)mv[c * 16 + i];
+    store_chunk(p, e, job, c, val, false, scale);
+  }
+  return true;
+}
+
+// 16-bit-lane path: tile sums fit int16, b_a <= 8, r = 0.  TMEM is read with two columns packed per
+// register (low half = even column); c - lo = relu(min(P - lo, hi - lo)) per lane in one instruction;
+// sums stay unsigned 16-bit lanes and are widened through the output buffer every flush_every tiles.
+__device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+  uint32_t S[EPI_COLS / 2];
+#pragma unroll
+  for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+  const uint32_t off = (uint32_t)(-p.lo);                    // c - lo lies in [0, hi - lo]
+  const uint32_t off2 = off | (off << 16);
+  const uint32_t rng2 = (uint32_t)(p.hi - p.lo) | ((uint32_t)(p.hi - p.lo) << 16);
+  int n_in_S = 0;
+  bool parked = false;   // int32 partial sums are parked in the output buffer
+  // Half of the warp's columns at a time through one load buffer; the other epilogue warp of the
+  // scheduler covers the load latency.
+  for (int ci = 0; ci < job.n_clamp_tiles; ++ci) {
+    const int buf = job.merging ? 1 : (ci & 1);
+    if (!mbar_wait(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+    uint32_t v[EPI_COLS / 4];
+    HDQT_LD_HALF_PACK(e.lane_addr + buf * BN, v);
+    HDQT_WAIT_HALF(v);
+#pragma unroll
+    for (int i = 0; i < EPI_COLS / 4; ++i) S[i] += __viaddmin_s16x2_relu(v[i], off2, rng2);
+    HDQT_LD_HALF_PACK(e.lane_addr + buf * BN + EPI_COLS / 2, v);
+    HDQT_WAIT_HALF(v);                                                 // the buffer is free
+    release_accumulator(e, buf, drains);
+#pragma unroll
+    for (int i = 0; i < EPI_COLS / 4; ++i) S[EPI_COLS / 4 + i] += __viaddmin_s16x2_relu(v[i], off2, rng2);
+    if (++n_in_S == p.flush_every && ci + 1 < job.n_clamp_tiles) {
+      // widen: park int32 partial sums in the output buffer
+      const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
+      const int64_t gn0 = (int64_t)job.n0 + e.grp * EPI_COLS;
+      const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+                       (gn0 + EPI_COLS <= p.N);
+      if (gm < p.M) {
+#pragma unroll
+        for (int i = 0; i < EPI_COLS / 2; i += 2) {
+          int s4[4];
+          s4[0] = (int)(S[i] & 0xFFFFu) - (int)off * n_in_S;
+          s4[1] = (int)(S[i] >> 16) - (int)off * n_in_S;
+          s4[2] = (int)(S[i + 1] & 0xFFFFu) - (int)off * n_in_S;
+          s4[3] = (int)(S[i + 1] >> 16) - (int)off * n_in_S;
+          emit4<false>(p, gm, gn0 + 2 * i, s4, parked, vec, 0.0f);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+      n_in_S = 0;
+      parked = true;
+    }
+  }
+  if (job.n_merged > 0) {
+    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+  }
+  const float scale = dequant_scale(p);
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) {
+    uint32_t mv[16];
+    if (job.n_merged > 0) {   // uniform
+      HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
+      HDQT_TMEM_WAIT16(mv);
+      // the last of the merged accumulator is in registers: hand it back to the MMA issuer
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drains);
+    }
+    int val[16];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t sp = S[c * 8 + i];
+      val[2 * i] = (int)(sp & 0xFFFFu) - (int)off * n_in_S;
+      val[2 * i + 1] = (int)(sp >> 16) - (int)off * n_in_S;
+      if (job.n_merged > 0) {
+        val[2 * i] += (int)mv[2 * i];
+        val[2 * i + 1] += (int)mv[2 * i + 1];
+      }
+    }
+    store_chunk(p, e, job, c, val, parked, scale);
+  }
+  return true;
+}
+
+// 32-bit path: one register per accumulator element, any b_a and shift r, optional per-tile debug output.
+template <bool kShift, bool kTilesOut>
+__device__ __forceinline__ bool epilogue_wide(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+  int S[EPI_COLS];
+#pragma unroll
+  for (int i = 0; i < EPI_COLS; ++i) S[i] = 0;
+  const int r = p.acc_shift, lo = p.lo, hi = p.hi;
+  for (int ci = 0; ci < job.n_clamp_tiles; ++ci) {
+    const int buf = job.merging ? 1 : (ci & 1);
+    if (!mbar_wait(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+#pragma unroll
+    for (int c = 0; c < EPI_COLS / 16; ++c) {
+      uint32_t v[16];
+      HDQT_TMEM_LD16(e.lane_addr + buf * BN + c * 16, v);
+      HDQT_TMEM_WAIT16(v);
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, buf, drains);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int ct = acc_quant<kShift>((int)v[i], r, lo, hi);
+        S[c * 16 + i] += ct;
+        if (kTilesOut) {
+          const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
+          const int64_t n = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16 + i;
+          if (gm < p.M && n < p.N) {
+            const int64_t o = ((int64_t)ci * p.M + gm) * p.N + n;
+            if (p.tiles_elem_bytes == 1) reinterpret_cast<int8_t*>(p.tiles_out)[o] = (int8_t)ct;
+            else reinterpret_cast<int16_t*>(p.tiles_out)[o] = (int16_t)ct;
+          }
+        }
+      }
+    }
+  }
+  if (job.n_merged > 0) {
+    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+    tc_fence_after();
+  }
+  const float scale = dequant_scale(p);
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 16; ++c) {
+    int val[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) val[i] = S[c * 16 + i];
+    if (job.n_merged > 0) {   // uniform
+      uint32_t mv[16];
+      HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
+      HDQT_TMEM_WAIT16(mv);
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drains);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) val[i] += (int)mv[i];
+    }
+    store_chunk(p, e, job, c, val, false, scale);
+  }
+  return true;
+}
+
+}  // namespace
+
+}  // namespace hdqt
