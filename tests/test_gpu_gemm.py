@@ -381,7 +381,8 @@ def test_persistent_ctas_mix_merged_and_clamped_blocks(hdqt):
         assert np.array_equal(out.cpu().numpy(), want_out), flags
 
 
-def test_work_split_pure_fixup_and_general_blocks(hdqt):
+@pytest.mark.parametrize("acc_bits,acc_tile", [(8, 32), (8, 64), (6, 32)])
+def test_work_split_pure_fixup_and_general_blocks(hdqt, acc_bits, acc_tile):
     """Large enough for the work split (>= 8 blocks per SM): pair blocks that are fully certified, that have a
     few uncertified tiles (fix-up pass) and that have many (general kernel), with ragged edges."""
     rng = np.random.default_rng(88)
@@ -396,14 +397,28 @@ def test_work_split_pure_fixup_and_general_blocks(hdqt):
     Bq[:, 320:352] = rng.integers(-8, 8, size=(N, 32))
     Bq[:, 1024:1056] = rng.integers(6, 8, size=(N, 32))      # large codes: these tiles really clamp
     Aq[2 * 128:3 * 128, 1024:1056] = rng.integers(6, 8, size=(128, 32))
-    want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 0.25, 0.5)
+    # the oracle on sampled rows (all columns) and sampled columns (all rows) keeps this test affordable
+    rows = np.sort(rng.choice(M, 96, replace=False))
+    cols = np.sort(rng.choice(N, 96, replace=False))
+    rows[:4] = [0, 2 * 128 + 5, M - 1, 128 * 5 + 7]          # incl. the really clamping block and the ragged edge
+    want_r, want_Sr, _ = O.gemm_i8_tiled(Aq[rows], Bq, 0.25, 0.5, acc_bits, acc_tile)
+    want_c, want_Sc, _ = O.gemm_i8_tiled(Aq, Bq[cols], 0.25, 0.5, acc_bits, acc_tile)
     na, nb = _dev(_tile_norms(Aq)), _dev(_tile_norms(Bq))
     qa, qb = torch.tensor([0.25], device="cuda"), torch.tensor([0.5], device="cuda")
     status = hdqt.new_status("cuda")
-    out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), qa, qb, want_S=True, norms_a=na, norms_b=nb, dev_status=status)
+    out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), qa, qb, acc_bits, acc_tile, want_S=True, norms_a=na,
+                                   norms_b=nb, dev_status=status)
     hdqt.check_device_status(status)
-    assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
-    assert np.array_equal(out.cpu().numpy(), want_out)
+    Sn, outn = S.cpu().numpy().astype(np.int64), out.cpu().numpy()
+    assert np.array_equal(Sn[rows], want_Sr) and np.array_equal(Sn[:, cols], want_Sc)
+    assert np.array_equal(outn[rows], want_r) and np.array_equal(outn[:, cols], want_c)
+    # the unsplit kernel (merging off) must give the same matrix everywhere
+    out2, S2, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), qa, qb, acc_bits, acc_tile, want_S=True, norms_a=na,
+                                     norms_b=nb, flags=hdqt.FLAG_NO_MERGE, dev_status=status)
+    hdqt.check_device_status(status)
+    assert torch.equal(S2, S) and torch.equal(out2, out)
+    if (acc_bits, acc_tile) != (8, 32):
+        return
     # the classes really occur: a fully certified pair block, one with a few uncertified tiles, one with many
     na64, nb64 = _tile_norms(Aq).astype(np.int64), _tile_norms(Bq).astype(np.int64)
     def uncert(tm, tn):
@@ -415,4 +430,5 @@ def test_work_split_pure_fixup_and_general_blocks(hdqt):
     # wide accumulators: every block goes to the pair kernel without certificates
     out16, S16, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), qa, qb, acc_bits=16, want_S=True, dev_status=status)
     hdqt.check_device_status(status)
-    assert np.array_equal(S16.cpu().numpy().astype(np.int64), Aq.astype(np.int64) @ Bq.astype(np.int64).T)
+    plain = np.rint(Aq.astype(np.float64) @ Bq.astype(np.float64).T).astype(np.int64)     # exact: small integers in fp64
+    assert np.array_equal(S16.cpu().numpy().astype(np.int64), plain)
