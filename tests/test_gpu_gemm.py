@@ -432,3 +432,28 @@ def test_work_split_pure_fixup_and_general_blocks(hdqt, acc_bits, acc_tile):
     hdqt.check_device_status(status)
     plain = np.rint(Aq.astype(np.float64) @ Bq.astype(np.float64).T).astype(np.int64)     # exact: small integers in fp64
     assert np.array_equal(S16.cpu().numpy().astype(np.int64), plain)
+
+
+def test_work_split_ragged_shapes_and_unaligned_output(hdqt):
+    """Split path with a single, half-empty row of pair blocks, a ragged last column block, a K that ends inside
+    a shared-memory stage, and an output whose leading dimension rules out vector stores."""
+    rng = np.random.default_rng(99)
+    M, N, K = 200, 256 * 1200 + 8, 96                        # 2 x 1201 single blocks >= 8 x 148
+    Aq = (rng.integers(-1, 2, size=(M, K)) * (rng.random((M, K)) < 0.2)).astype(np.int8)
+    Bq = (rng.integers(-1, 2, size=(N, K)) * (rng.random((N, K)) < 0.2)).astype(np.int8)
+    Bq[256 * 7:256 * 9, 32:64] = rng.integers(6, 8, size=(512, 32))      # a few blocks with one clamping tile
+    Aq[:, 32:64] = rng.integers(5, 8, size=(M, 32))
+    Bq[256 * 40:256 * 41] = rng.integers(-8, 8, size=(256, K))          # one block where nothing certifies
+    Aq[:, 64:96] = np.where(Aq[:, 64:96] == 0, 2, Aq[:, 64:96])
+    want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 0.5, 0.5)
+    na, nb = _dev(_tile_norms(Aq)), _dev(_tile_norms(Bq))
+    half = torch.tensor([0.5], device="cuda")
+    status = hdqt.new_status("cuda")
+    big = torch.full((M, N + 3), -7.0, device="cuda")
+    for view in (None, big[:, 1:N + 1]):
+        out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), half, half, want_S=True, norms_a=na, norms_b=nb,
+                                       dev_status=status, out=view)
+        hdqt.check_device_status(status)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
+        assert np.array_equal(out.cpu().numpy(), want_out)
+    assert (big[:, 0] == -7.0).all().item() and (big[:, N + 1:] == -7.0).all().item()
