@@ -15,7 +15,7 @@
 //                          clamp-free certificates of the next block, 8 epilogue warps drain the accumulators,
 //                          apply the accumulator quantisation per tile and keep the wide sums in registers
 //   hdqt_gemm_pair.cuh     large problems: block classification, cta_group::2 kernel for certified 256 x 256
-//                          blocks, CUDA-core fix-up of blocks with a few uncertified tiles
+//                          blocks, fix-up pass for blocks with a few uncertified tiles
 // Tiles that provably cannot clamp (Cauchy-Schwarz bound from per-tile code norms) may be
 // accumulated together in TMEM: the clamp is the identity there, so the integers are unchanged.
 // Every wait is bounded; when one runs out the CTA records HDQT_ERR_TIMEOUT and leaves.

@@ -82,6 +82,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   const int num_tiles = (p.block_list != nullptr) ? __ldg(p.block_count) : tiles_m * tiles_n;
   const int num_kblocks = (p.tiles32 + 3) >> 2;
   const int num_acc = p.num_acc;
+  if (num_tiles == 0) return;   // an empty work list (uniform over the grid): nothing to set up or tear down
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {

@@ -1,5 +1,5 @@
 // Work split for large problems: classification of 256 x 256 pair blocks, the cta_group::2 kernel for blocks
-// whose tiles are (nearly) all certified clamp-free, and the CUDA-core fix-up pass.  Included by hdqt_gemm.cu.
+// whose tiles are (nearly) all certified clamp-free, and the fix-up pass for their few uncertified tiles.  Included by hdqt_gemm.cu.
 #pragma once
 
 #include "hdqt_gemm_device.cuh"
@@ -344,14 +344,15 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 // ---- fix-up pass for pair blocks with a few uncertified accumulator tiles -----------------------------
 // The pair kernel accumulated ALL their tiles unclamped and parked the integer sums in the output buffer.
 // For an uncertified tile the accumulator quantisation may change the tile sum, so this pass recomputes
-// exactly those tile sums P on the CUDA cores and adds clamp(P) - P; the result is sum_t clamp(P_t) bit for bit
-// (on certified tiles the clamp is the identity).  Then it applies the dequantising scale.
+// exactly those tile sums P (warp-level mma.sync m16n8k32 on staged 32-byte K slices) and adds clamp(P) - P;
+// the result is sum_t clamp(P_t) bit for bit (on certified tiles the clamp is the identity).  Then it applies
+// the dequantising scale.
 // Work item = 64 rows of a 256 x 256 block (4 items per block, so that the few blocks spread over all SMs),
-// 256 threads: warp w owns rows 8w..8w+7, lane l owns the columns l + 32 j.  Corrections are rare, so they are
-// added to the parked sums in place as they are found.
+// 256 threads.  Corrections are rare, so they are added to the parked sums in place as they are found; the
+// final conversion walks the item with warp w on rows 8w..8w+7 and lane l on the columns l + 32 j.
 constexpr int FIX_ROWS = 64;
 constexpr int kMaxFixTiles = 256;   // the classification sends blocks with more uncertified tiles to the general kernel
-constexpr int FIX_B_STRIDE = 36;    // bytes per staged B row (32 + 4: consecutive rows fall into different banks)
+constexpr int FIX_B_STRIDE = 48;    // bytes per staged B row (32 + 16: the fragment loads of 8 rows x 4 lanes hit 32 banks)
 
 __global__ void __launch_bounds__(256, 2)
 fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict__ Bq, const GemmParams p,
@@ -391,11 +392,15 @@ fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict
     for (int u = 0; u < n_uncert; ++u) {
       const int a = s_list[u];
       const int t0 = a * p.tiles_per_acc, t1 = min(p.tiles32, t0 + p.tiles_per_acc);
-      int P[8][8];
+      // exact tile sums on the (legacy) int8 tensor path: warp w owns rows 16 (w & 3) .. +15 and the 128
+      // columns of half (w >> 2), as 16 m16n8k32 tiles; C[nt] = rows (g, g + 8) x columns 8 nt + 2 tig, + 1
+      int Cf[16][4];
 #pragma unroll
-      for (int r = 0; r < 8; ++r)
+      for (int nt = 0; nt < 16; ++nt)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) P[r][j] = 0;
+        for (int i = 0; i < 4; ++i) Cf[nt][i] = 0;
+      const int g = lane >> 2, tig = lane & 3;
+      const int arow = (warp & 3) * 16 + g, col_half = (warp >> 2) * 128;
       for (int t = t0; t < t1; ++t) {
         __syncthreads();
         {   // stage the 32-byte K slice of 64 rows of A and 256 rows of B (rows beyond the matrices read as zero)
@@ -408,32 +413,34 @@ fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict
             const int brow = row + FIX_ROWS * h;
             uint2 vb = make_uint2(0u, 0u);
             if (n0 + brow < p.N) vb = __ldg(reinterpret_cast<const uint2*>(Bq + (n0 + brow) * p.K_pad + (int64_t)t * 32 + part * 8));
-            uint32_t* db = reinterpret_cast<uint32_t*>(sB + brow * FIX_B_STRIDE + part * 8);
-            db[0] = vb.x;
-            db[1] = vb.y;
+            *reinterpret_cast<uint2*>(sB + brow * FIX_B_STRIDE + part * 8) = vb;
           }
         }
         __syncthreads();
+        // A fragment: (row g, k 4 tig..), (row g + 8, same k), then the same rows at k + 16
+        const int a0 = *reinterpret_cast<const int*>(sA + arow * 32 + tig * 4);
+        const int a1 = *reinterpret_cast<const int*>(sA + (arow + 8) * 32 + tig * 4);
+        const int a2 = *reinterpret_cast<const int*>(sA + arow * 32 + 16 + tig * 4);
+        const int a3 = *reinterpret_cast<const int*>(sA + (arow + 8) * 32 + 16 + tig * 4);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          int av[8], bv[8];
-#pragma unroll
-          for (int r = 0; r < 8; ++r) av[r] = *reinterpret_cast<const int*>(sA + (warp * 8 + r) * 32 + k * 4);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) bv[j] = *reinterpret_cast<const int*>(sB + (lane + 32 * j) * FIX_B_STRIDE + k * 4);
-#pragma unroll
-          for (int r = 0; r < 8; ++r)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) P[r][j] = __dp4a(av[r], bv[j], P[r][j]);
+        for (int nt = 0; nt < 16; ++nt) {
+          // B fragment: column n = 8 nt + g of the tile (= row n of the code matrix), k 4 tig.. and k + 16
+          const uint8_t* brow = sB + (col_half + nt * 8 + g) * FIX_B_STRIDE;
+          const int b0 = *reinterpret_cast<const int*>(brow + tig * 4);
+          const int b1 = *reinterpret_cast<const int*>(brow + 16 + tig * 4);
+          asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                       : "+r"(Cf[nt][0]), "+r"(Cf[nt][1]), "+r"(Cf[nt][2]), "+r"(Cf[nt][3])
+                       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
         }
       }
 #pragma unroll
-      for (int r = 0; r < 8; ++r) {
-        const int64_t gm = m0 + warp * 8 + r;
+      for (int nt = 0; nt < 16; ++nt) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int64_t gn = n0 + lane + 32 * j;
-          const int d = min(max(P[r][j], p.lo), p.hi) - P[r][j];
+        for (int i = 0; i < 4; ++i) {
+          const int64_t gm = m0 + arow + (i >> 1) * 8;
+          const int64_t gn = n0 + col_half + nt * 8 + tig * 2 + (i & 1);
+          const int P = Cf[nt][i];
+          const int d = min(max(P, p.lo), p.hi) - P;
           if (d != 0 && gm < p.M && gn < p.N) {
             int* o = reinterpret_cast<int*>(p.out + gm * p.ld_out + gn);   // only this thread touches this element
             *o += d;
@@ -441,6 +448,7 @@ fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict
         }
       }
     }
+    __syncthreads();   // the corrections above and the conversion below use different thread-to-element maps
     // parked (now exact) integer sums -> fp32, lanes on consecutive columns; all loads first, so that
     // they are in flight together (each element is touched by this thread only)
     int Sv[8][8];
