@@ -22,19 +22,35 @@ struct Philox4 {
   uint32_t w[4];
 };
 
+// The ten round keys of Philox4x32-10 depend on the seed only: the host computes them once per launch and
+// passes them as a kernel parameter, so the kernels spend no instructions on the key schedule.
+struct PhiloxKeys {
+  uint32_t k[10][2];
+};
+
+inline PhiloxKeys make_philox_keys(uint64_t seed) {
+  PhiloxKeys keys;
+  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    keys.k[r][0] = k0;
+    keys.k[r][1] = k1;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return keys;
+}
+
 __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                                 uint32_t k0, uint32_t k1) {
-  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+                                                 const PhiloxKeys& keys) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
     const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
     const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
-    c0 = hi1 ^ c1 ^ k0;
+    c0 = hi1 ^ c1 ^ keys.k[r][0];
     c1 = lo1;
-    c2 = hi0 ^ c3 ^ k1;
+    c2 = hi0 ^ c3 ^ keys.k[r][1];
     c3 = lo0;
-    k0 += W0;
-    k1 += W1;
   }
   Philox4 o;
   o.w[0] = c0; o.w[1] = c1; o.w[2] = c2; o.w[3] = c3;

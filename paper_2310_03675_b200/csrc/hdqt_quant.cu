@@ -119,7 +119,8 @@ struct QuantParams {
   int lo, hi;
   int mode;          // hdqt_round_t
   bool sr_magic;     // |v| < 64 guaranteed: fixed-point conversion through the fp32 adder
-  uint32_t k0, k1, tag;
+  uint32_t tag;
+  const PhiloxKeys* keys;   // the launch's round keys (a kernel parameter)
 };
 
 // codes of 8 consecutive elements; `g` = (linear index of the first element) / 8
@@ -134,7 +135,7 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams
       c[i] = min(max(q, p.lo), p.hi);
     }
   } else {
-    const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, 0u, p.k0, p.k1);
+    const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, 0u, *p.keys);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float v = __fmul_rn(x[i], p.m);
@@ -159,15 +160,14 @@ __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
 }
 
 __device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bits, float clip, int mode,
-                                                   uint64_t seed, uint32_t tag) {
+                                                   const PhiloxKeys* keys, uint32_t tag) {
   QuantParams p;
   p.m = qs.m;
   p.lo = -(1 << (bits - 1));
   p.hi = (1 << (bits - 1)) - 1;
   p.mode = mode;
   p.sr_magic = ((float)(1 << (bits - 1)) <= 32.0f * clip);  // |v| <= 32 (1 + eps)
-  p.k0 = (uint32_t)seed;
-  p.k1 = (uint32_t)(seed >> 32);
+  p.keys = keys;
   p.tag = tag;
   return p;
 }
@@ -257,11 +257,12 @@ absmax_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t
 
 __global__ void __launch_bounds__(kThreads)
 quantize_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_row, int64_t K_pad,
-                   int had_block, bool vec, int bits, float clip, int mode, uint64_t seed, uint32_t tag,
+                   int had_block, bool vec, int bits, float clip, int mode,
+                   const __grid_constant__ PhiloxKeys keys, uint32_t tag,
                    const float* __restrict__ amax_ptr, int8_t* __restrict__ codes, float* step_out,
                    uint16_t* __restrict__ row_norms, int32_t* dev_status) {
   const QuantScale qs = make_quant_scale(__ldg(amax_ptr), clip, bits);
-  const QuantParams p = make_params(qs, bits, clip, mode, seed, tag);
+  const QuantParams p = make_params(qs, bits, clip, mode, &keys, tag);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     *step_out = qs.step;
     if (qs.bad) report_status(dev_status, HDQT_ERR_NONFINITE);
@@ -385,12 +386,13 @@ absmax_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t
 
 __global__ void __launch_bounds__(kThreads, 3)
 quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_k, int64_t K_pad,
-                   int had_block, int bits, float clip, int mode, uint64_t seed, uint32_t tag,
+                   int had_block, int bits, float clip, int mode,
+                   const __grid_constant__ PhiloxKeys keys, uint32_t tag,
                    const float* __restrict__ amax_ptr, int8_t* __restrict__ codes, float* step_out,
                    int32_t* __restrict__ tile_norms, int32_t* dev_status) {
   __shared__ int s_norm[kThreads / 32];
   const QuantScale qs = make_quant_scale(__ldg(amax_ptr), clip, bits);
-  const QuantParams p = make_params(qs, bits, clip, mode, seed, tag);
+  const QuantParams p = make_params(qs, bits, clip, mode, &keys, tag);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     *step_out = qs.step;
     if (qs.bad) report_status(dev_status, HDQT_ERR_NONFINITE);
@@ -495,12 +497,13 @@ hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t
                               cudaStream_t s) {
   const int64_t K_pad = hdqt_padded_k(K, had_block);
   const int64_t T = K_pad >> 5;
+  const PhiloxKeys keys = make_philox_keys(seed);
   if (ld_k == 1) {
     const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
     const int64_t total = rows * (K_pad >> 3);
     uint16_t* rn = tile_norms ? row_norms_scratch : nullptr;
     quantize_kc_kernel<<<grid_for(total, kThreads * kUnrollQuant, 4), kThreads, 0, s>>>(
-        src, rows, K, ld_row, K_pad, had_block, vec, bits, clip, mode, seed, tag, amax, codes, step_out, rn,
+        src, rows, K, ld_row, K_pad, had_block, vec, bits, clip, mode, keys, tag, amax, codes, step_out, rn,
         dev_status);
     if (tile_norms) {
       dim3 grid((unsigned)((T + 63) / 64), (unsigned)((rows + 127) / 128));
@@ -510,7 +513,7 @@ hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t
     const int64_t items = ((rows + kThreads - 1) / kThreads) * T;
     if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
     quantize_ks_kernel<<<grid_for(items, 1, 3), kThreads, 0, s>>>(
-        src, rows, K, ld_k, K_pad, had_block, bits, clip, mode, seed, tag, amax, codes, step_out, tile_norms,
+        src, rows, K, ld_k, K_pad, had_block, bits, clip, mode, keys, tag, amax, codes, step_out, tile_norms,
         dev_status);
   }
   return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
