@@ -143,7 +143,8 @@ hdqt_status_t hdqt_absmax_hadamard(const float* src, int64_t rows, int64_t K,
  *           rows and every 32-wide K tile, max over the rows of sum(code^2); lets
  *           the GEMM prove that a tile cannot clamp.  NULL = not produced.
  * workspace: at least hdqt_quantize_workspace_bytes(rows, K, had_block) bytes (holds the
- *           measured maximum and per-row tile norms).
+ *           measured maximum and the partial maxima the calibration pass hands to the
+ *           quantize pass).
  */
 hdqt_status_t hdqt_quantize_hadamard(const float* src, int64_t rows, int64_t K,
                                      int64_t ld_row, int64_t ld_k, int32_t had_block,
@@ -170,19 +171,22 @@ size_t hdqt_quantize_workspace_bytes(int64_t rows, int64_t K, int32_t had_block)
  * caller's buffers.
  *
  * Limits and rules
- *   - The array is HDQT_STATIC_SCRATCH_BYTES (4 MiB + 256 B) and exists once per GPU for as long
- *     as the library stays loaded.  It must hold 2 bytes per (row, 32-wide K tile):
- *     rows * (K_pad / 32) <= 2 097 152 (e.g. 8192 x 8192).  Larger operands are refused with
- *     HDQT_ERR_STATIC_SCRATCH and nothing is launched; use hdqt_quantize_hadamard then.
+ *   - The array is HDQT_STATIC_SCRATCH_BYTES and exists once per GPU for as long as the library
+ *     stays loaded.  It holds the measured maximum and the partial maxima that the calibration
+ *     pass leaves for the quantize pass (one per thread block of that pass).
+ *   - Stated maximum operand size: rows * (K_pad / 32) <= HDQT_STATIC_MAX_ROW_TILES (2 097 152,
+ *     e.g. 8192 x 8192).  Larger operands are refused with HDQT_ERR_STATIC_SCRATCH and nothing is
+ *     launched; use hdqt_quantize_hadamard then.
  *   - The first call on each device looks up the array's device address (a cheap runtime query,
  *     made with that device current); make that first call during set-up, before any stream
  *     capture you may do.
  *   - All calls on a device share the one array, and it keeps what the previous call left in it.
- *     Each call re-initialises the parts that must start from zero, so back-to-back calls on one
+ *     Every entry a call reads is written by that same call first, so back-to-back calls on one
  *     stream are fine; calls that can overlap on the GPU (different streams, no ordering between
  *     them) race on the array and corrupt each other's results.
  */
-#define HDQT_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u + 256u)
+#define HDQT_STATIC_SCRATCH_BYTES (256u + 4096u)
+#define HDQT_STATIC_MAX_ROW_TILES 2097152
 
 hdqt_status_t hdqt_quantize_hadamard_static(const float* src, int64_t rows, int64_t K,
                                             int64_t ld_row, int64_t ld_k, int32_t had_block,
@@ -241,6 +245,16 @@ hdqt_status_t hdqt_calibrate_acc_shift(const int8_t* Aq, const int8_t* Bq, int64
                                        int32_t acc_tile, int32_t* shift_out,
                                        void* workspace, size_t workspace_bytes,
                                        int32_t* dev_status, void* stream);
+
+/*
+ * Diagnostic: runs the two bounded barrier waits that the GEMM kernels use (Section 3's tiled matmul is
+ * a producer/consumer pipeline here) on a barrier nothing arrives at, with a budget of about a
+ * millisecond, in a one-block kernel with no copy or tensor-core operation in flight.  Every waiting
+ * thread must give up and the block must end normally: afterwards *dev_status holds HDQT_ERR_TIMEOUT
+ * (sticky maximum, as for the GEMM kernels) and *gave_up (optional device int32, the caller zeroes it)
+ * the number of threads whose wait ran out (1 spinning thread + 32 suspending ones).
+ */
+hdqt_status_t hdqt_selftest_bounded_wait(int32_t* dev_status, int32_t* gave_up, void* stream);
 
 /* ------------------------------------------------------------------------ */
 /* The three training GEMMs of one linear layer (Section 3: Z = X W and the    */

@@ -22,6 +22,8 @@ hdqt_status_t check_quant_args(const float* src, int64_t rows, int64_t K, int64_
   return HDQT_OK;
 }
 
+constexpr int64_t kMinBlocksForNorms = 32;
+
 struct OperandView {  // logical [rows, K] view of an operand with the contraction index as "K"
   const float* src;
   int64_t rows, ld_row, ld_k;
@@ -82,11 +84,10 @@ extern "C" hdqt_status_t hdqt_absmax_hadamard(const float* src, int64_t rows, in
                        reinterpret_cast<cudaStream_t>(stream));
 }
 
-// workspace of hdqt_quantize_hadamard: [amax fp32 | pad to 256 | per-row tile norms u16 [rows, K_pad/32]]
+// workspace of hdqt_quantize_hadamard: [measured maximum fp32 | pad to 256 | partial maxima u32[kMaxPartials]]
 extern "C" size_t hdqt_quantize_workspace_bytes(int64_t rows, int64_t K, int32_t had_block) {
   if (rows <= 0 || K <= 0 || had_block < 1) return 0;
-  const int64_t T = hdqt_padded_k(K, had_block) / 32;
-  return 256 + align_up((size_t)rows * (size_t)T * sizeof(uint16_t), 256);
+  return 256 + sizeof(uint32_t) * (size_t)kMaxPartials;
 }
 
 extern "C" hdqt_status_t hdqt_quantize_hadamard(const float* src, int64_t rows, int64_t K, int64_t ld_row,
@@ -104,17 +105,15 @@ extern "C" hdqt_status_t hdqt_quantize_hadamard(const float* src, int64_t rows, 
   if ((reinterpret_cast<uintptr_t>(codes) & 127) || (reinterpret_cast<uintptr_t>(workspace) & 127))
     return HDQT_ERR_ALIGNMENT;
   if (workspace_bytes < hdqt_quantize_workspace_bytes(rows, K, had_block)) return HDQT_ERR_WORKSPACE;
-  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  float* amax_ws = reinterpret_cast<float*>(workspace);
-  uint16_t* row_norms = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(workspace) + 256);
-  const float* amax = amax_in;
-  if (amax == nullptr) {
-    st = launch_absmax(src, rows, K, ld_row, ld_k, had_block, amax_ws, dev_status, s);
-    if (st != HDQT_OK) return st;
-    amax = amax_ws;
-  }
-  return launch_quantize(src, rows, K, ld_row, ld_k, had_block, bits, clip, mode, seed, tag, amax, codes,
-                         step_out, tile_norms, row_norms, dev_status, s);
+  QuantOperand a{};
+  a.src = src; a.rows = rows; a.K = K; a.ld_row = ld_row; a.ld_k = ld_k;
+  a.clip = clip; a.mode = mode; a.tag = tag;
+  a.amax_in = amax_in;
+  a.amax_slot = reinterpret_cast<float*>(workspace);
+  a.codes = codes; a.step_out = step_out; a.tile_norms = tile_norms;
+  return launch_calibrate_quantize(&a, 1, had_block, bits, seed,
+                                   reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(workspace) + 256),
+                                   dev_status, reinterpret_cast<cudaStream_t>(stream));
 }
 
 // ---- the three training GEMMs -----------------------------------------------------------------
@@ -136,7 +135,7 @@ extern "C" hdqt_status_t hdqt_workspace_layout(const hdqt_gemm_desc_t* d, int64_
   out->norms_a = off; off += align_up((size_t)((M + 127) / 128) * T * sizeof(int32_t), 256);
   out->norms_b = off; off += align_up((size_t)((N + 127) / 128) * T * sizeof(int32_t), 256);
   out->gemm_ws = off;
-  const size_t quant_ws = hdqt_quantize_workspace_bytes(M > N ? M : N, K, d->had_block);
+  const size_t quant_ws = 2 * sizeof(uint32_t) * (size_t)kMaxPartials;   // partial maxima of both operands
   const size_t gemm_ws = hdqt_gemm_i8_workspace_bytes(M, N, K_pad);
   off += align_up(quant_ws > gemm_ws ? quant_ws : gemm_ws, 256);
   out->total = off;
@@ -174,7 +173,20 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
   const uint32_t tagA = swap ? d->tag_b : d->tag_a, tagB = swap ? d->tag_a : d->tag_b;
   const float* amaxA = swap ? d->amax_b : d->amax_a;
   const float* amaxB = swap ? d->amax_a : d->amax_b;
-  const bool merge = !(d->flags & HDQT_FLAG_NO_MERGE) && d->acc_shift == 0;
+  // Tile norms are worth producing only where the GEMM can use them: merging allowed, a tile sum that can
+  // exceed the accumulator at all, and enough output blocks for the merged path to pay for the blocked
+  // quantize mapping (small products are bound by launch latency, not by the accumulator epilogue).
+  bool merge = !(d->flags & HDQT_FLAG_NO_MERGE) && d->acc_shift == 0 && d->acc_bits >= 2 && d->acc_bits < 32 &&
+               d->in_bits >= 2 && d->in_bits <= 8 && d->acc_tile >= 0;
+  if (merge) {
+    const int64_t tiles32 = L.k_pad / 32;
+    const int64_t tpa = d->acc_tile == 0 ? tiles32 : d->acc_tile / 32;
+    const int64_t code_max = int64_t(1) << (d->in_bits - 1);
+    const int64_t p_max = tpa * 32 * code_max * code_max;
+    const int64_t hi = (int64_t(1) << (d->acc_bits - 1)) - 1;
+    const int64_t blocks = ((M + 127) / 128) * ((N + 255) / 256);
+    merge = (p_max > hi) && (blocks >= kMinBlocksForNorms);
+  }
   int32_t* normsA = merge ? reinterpret_cast<int32_t*>(ws + L.norms_a) : nullptr;
   int32_t* normsB = merge ? reinterpret_cast<int32_t*>(ws + L.norms_b) : nullptr;
   const size_t scratch_bytes = L.total - L.gemm_ws;
@@ -190,29 +202,18 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
     return HDQT_ERR_INVALID_ARG;
 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  // measured maxima live where the layout says (harnesses read them back); both are cleared by one memset
-  float* amax_slot_a = reinterpret_cast<float*>(ws + L.amax_a);
-  float* amax_slot_b = reinterpret_cast<float*>(ws + L.amax_b);
-  if (!amaxA || !amaxB) {
-    if (cudaMemsetAsync(ws + L.amax_a, 0, (L.amax_b - L.amax_a) + sizeof(float), s) != cudaSuccess) return HDQT_ERR_CUDA;
-  }
-  uint16_t* row_norms = reinterpret_cast<uint16_t*>(ws + L.gemm_ws);
-  if (scratch_bytes < hdqt_quantize_workspace_bytes(M > N ? M : N, K, d->had_block)) return HDQT_ERR_WORKSPACE;
-  if (!amaxA) {
-    st = launch_absmax(gA.src, gA.rows, K, gA.ld_row, gA.ld_k, d->had_block, amax_slot_a, dev_status, s, false);
-    if (st != HDQT_OK) return st;
-  }
-  if (!amaxB) {
-    st = launch_absmax(gB.src, gB.rows, K, gB.ld_row, gB.ld_k, d->had_block, amax_slot_b, dev_status, s, false);
-    if (st != HDQT_OK) return st;
-  }
-  st = launch_quantize(gA.src, gA.rows, K, gA.ld_row, gA.ld_k, d->had_block, d->in_bits, clipA, roundA, d->seed, tagA,
-                       amaxA ? amaxA : amax_slot_a, reinterpret_cast<int8_t*>(ws + L.codes_a),
-                       reinterpret_cast<float*>(ws + L.step_a), normsA, row_norms, dev_status, s);
-  if (st != HDQT_OK) return st;
-  st = launch_quantize(gB.src, gB.rows, K, gB.ld_row, gB.ld_k, d->had_block, d->in_bits, clipB, roundB, d->seed, tagB,
-                       amaxB ? amaxB : amax_slot_b, reinterpret_cast<int8_t*>(ws + L.codes_b),
-                       reinterpret_cast<float*>(ws + L.step_b), normsB, row_norms, dev_status, s);
+  if (scratch_bytes < 2 * sizeof(uint32_t) * (size_t)kMaxPartials) return HDQT_ERR_WORKSPACE;
+  // both operands in one calibration and one quantize launch (per memory layout); measured maxima are
+  // published where the layout says (harnesses read them back)
+  QuantOperand ops[2];
+  ops[0] = QuantOperand{gA.src, gA.rows, K, gA.ld_row, gA.ld_k, clipA, roundA, tagA, amaxA,
+                        reinterpret_cast<float*>(ws + L.amax_a), reinterpret_cast<int8_t*>(ws + L.codes_a),
+                        reinterpret_cast<float*>(ws + L.step_a), normsA};
+  ops[1] = QuantOperand{gB.src, gB.rows, K, gB.ld_row, gB.ld_k, clipB, roundB, tagB, amaxB,
+                        reinterpret_cast<float*>(ws + L.amax_b), reinterpret_cast<int8_t*>(ws + L.codes_b),
+                        reinterpret_cast<float*>(ws + L.step_b), normsB};
+  st = launch_calibrate_quantize(ops, 2, d->had_block, d->in_bits, d->seed,
+                                 reinterpret_cast<uint32_t*>(ws + L.gemm_ws), dev_status, s);
   if (st != HDQT_OK) return st;
   return hdqt_gemm_i8_tiled(reinterpret_cast<int8_t*>(ws + L.codes_a), reinterpret_cast<int8_t*>(ws + L.codes_b),
                             reinterpret_cast<float*>(ws + L.step_a), reinterpret_cast<float*>(ws + L.step_b), M, N,

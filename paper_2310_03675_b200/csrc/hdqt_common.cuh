@@ -84,17 +84,33 @@ inline hdqt_status_t cuda_failure(cudaError_t e, const char* what) {
 }
 
 // ---- internal launchers (defined in the .cu files) ----
-// zero_first = false: the caller has already cleared *amax_out on the stream
+
+constexpr int kMaxPartials = 1024;   // partial calibration maxima per operand (>= thread blocks of a calibration launch)
+
+// One operand of a transform + quantize call: logical [rows, K], element (r, k) = src[r*ld_row + k*ld_k].
+struct QuantOperand {
+  const float* src;
+  int64_t rows, K, ld_row, ld_k;
+  float clip;
+  int32_t mode;          // hdqt_round_t
+  uint32_t tag;
+  const float* amax_in;  // supplied calibration maximum (device) or nullptr = measure
+  float* amax_slot;      // optional: where the measured maximum is published
+  int8_t* codes;
+  float* step_out;
+  int32_t* tile_norms;   // optional
+};
+
+// amax_out[0] = max |src H| (zeroes amax_out first, then one launch)
 hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
-                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s,
-                            bool zero_first = true);
+                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s);
 
-hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
-                              int32_t had_block, int32_t bits, float clip, int32_t mode, uint64_t seed,
-                              uint32_t tag, const float* amax, int8_t* codes, float* step_out,
-                              int32_t* tile_norms, uint16_t* row_norms_scratch, int32_t* dev_status,
-                              cudaStream_t s);
+// Calibration (for operands without a supplied maximum) and quantize passes for one or two operands that
+// share had_block, bits and seed: at most one launch per pass and memory layout.
+// partials: scratch of n_ops * kMaxPartials uint32.
+hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int32_t had_block, int32_t bits,
+                                        uint64_t seed, uint32_t* partials, int32_t* dev_status, cudaStream_t s);
 
-int sm_count();
+int sm_count();   // of the current device
 
 }  // namespace hdqt

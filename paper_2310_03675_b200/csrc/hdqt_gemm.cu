@@ -58,6 +58,28 @@ __global__ void calibrate_shift_kernel(const int8_t* __restrict__ Aq, const int8
   if ((threadIdx.x & 31) == 0 && need > 0) atomicMax(shift_out, need);
 }
 
+// ---- self-test of the bounded waits ------------------------------------------------------------
+// Both wait forms of the GEMM kernels, on a barrier that nothing ever arrives at, with a poll budget of about a
+// millisecond instead of the kernels' second: each must give up, raise the block's abort flag and let the
+// block end normally with HDQT_ERR_TIMEOUT in the status word.  No TMA copy or tensor-core operation is in
+// flight, so there is nothing to drain.
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(int32_t* dev_status, int32_t* gave_up) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, 1 << 10);          // spin, then back off
+  if (threadIdx.x >= 32) ok = mbar_wait_yield<64>(smem_u32(&bar), 0u, &abort_flag, 1 << 12);   // suspend and sleep
+  if (!ok && gave_up != nullptr) atomicAdd(gave_up, 1);
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag) report_status(dev_status, HDQT_ERR_TIMEOUT);
+}
+
 // ---- host side --------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -188,7 +210,9 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
   p.dev_status = dev_status;
 
   // 16-bit-lane epilogue: tile sums fit int16, the offset sums fit uint16 for flush_every tiles
-  const bool packed = !tiles_out && acc_shift == 0 && acc_bits <= 8 && p_max <= 32767;
+  // (the epilogue forms P + 2^(b_a-1) in signed 16-bit lanes before it takes the minimum)
+  const bool packed = !tiles_out && acc_shift == 0 && acc_bits <= 8 && p_max + ((int64_t)p.hi + 1) <= 32767;
+  p.offset_mma = packed ? 1 : 0;
   p.flush_every = packed ? (int32_t)(65535 / ((int64_t)p.hi - p.lo)) : 0;
   if (p.flush_every > 256) p.flush_every = 256;
 
@@ -281,3 +305,16 @@ extern "C" hdqt_status_t hdqt_calibrate_acc_shift(const int8_t* Aq, const int8_t
                                                                        shift_out);
   return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
 }
+
+extern "C" hdqt_status_t hdqt_selftest_bounded_wait(int32_t* dev_status, int32_t* gave_up, void* stream) {
+  if (!dev_status) return HDQT_ERR_INVALID_ARG;
+  bounded_wait_selftest_kernel<<<1, 64, 0, reinterpret_cast<cudaStream_t>(stream)>>>(dev_status, gave_up);
+  return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
+}
+
+#ifdef HDQT_TIMELINE
+// tuning builds only: copies the recorded event timeline (64 tiles x 16 slots of SM clock values) to the host
+extern "C" int hdqt_debug_timeline(long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_timeline, sizeof(long long) * 64 * 16);
+}
+#endif

@@ -21,7 +21,13 @@ constexpr int B_STAGE = BN * BKB;              // 32 KB
 constexpr int STAGE_BYTES = A_STAGE + B_STAGE; // 48 KB
 constexpr int NUM_EPI_WARPS = 8;               // 2 per TMEM lane quarter, 128 accumulator columns each
 constexpr int EPI_COLS = BN / (NUM_EPI_WARPS / 4);
-constexpr int GEMM_THREADS = 32 * (3 + NUM_EPI_WARPS);   // + TMA producer, MMA issuer, certificate builder
+constexpr int NUM_CTRL_WARPS = 4;   // warp group 0: TMA producer, MMA issuer, certificate builder, one spare
+constexpr int GEMM_THREADS = 32 * (NUM_CTRL_WARPS + NUM_EPI_WARPS);
+// Register split between the warp groups (setmaxnreg): the kernel is compiled for 168 registers per thread
+// (384 threads), the control warps give most of theirs back and the epilogue warps take them:
+// 128 * 72 + 256 * 216 = 384 * 168.
+constexpr int CTRL_REGS = 72;
+constexpr int EPI_REGS = 216;
 constexpr int TMEM_COLS = 512;
 constexpr int MAX_CERT_WORDS = 256;            // certificate bitmask: up to 8192 accumulator tiles
 constexpr int OUT_STAGE_WARP = 32 * 16 * 4;    // per epilogue warp: a 32-row x 16-column fp32 box for the store transpose
@@ -29,13 +35,37 @@ constexpr int TILE_INFO_BYTES = 4 * MAX_CERT_WORDS + 16;
 // the dynamic shared-memory window is declared 1024-byte aligned (checked in the kernel), so no slack is kept
 // offset of the store boxes (128-byte aligned)
 constexpr int OUT_STAGE_OFF = (STAGES * STAGE_BYTES + 256 /*barriers*/ + 2 * TILE_INFO_BYTES + 127) / 128 * 128;
-constexpr int SMEM_BYTES = OUT_STAGE_OFF + NUM_EPI_WARPS * OUT_STAGE_WARP;
+// constant operand tiles of the offset MMA (see epilogue_packed): no swizzle, 8-row groups 256 bytes apart,
+// the two 16-byte K chunks of a row group 128 bytes apart
+constexpr int OFFS_A_OFF = OUT_STAGE_OFF + NUM_EPI_WARPS * OUT_STAGE_WARP;
+constexpr int OFFS_A_BYTES = (BM / 8) * 256;   // 4 KB
+constexpr int OFFS_B_OFF = OFFS_A_OFF + OFFS_A_BYTES;
+constexpr int OFFS_B_BYTES = (BN / 8) * 256;   // 8 KB
+constexpr int SMEM_BYTES = OFFS_B_OFF + OFFS_B_BYTES;
 static_assert(OUT_STAGE_WARP % 128 == 0, "store boxes must stay 128-byte aligned");
 static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
 // instruction descriptor: D = s32, A = B = signed 8-bit, both K-major, N = 256, M = 128
 constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                            ((uint32_t)(BM >> 4) << 24);
+
+// Optional event timeline for kernel tuning (compiled in only with -DHDQT_TIMELINE): block 0 records the
+// SM clock at a few points of its first 64 accumulator tiles into a device array that
+// hdqt_debug_timeline copies out.  Slots: 0 MMA issuer got the accumulator, 1 MMA issuer committed the tile,
+// 2 epilogue saw the tile, 4 accumulator released, 5 tile added up (first epilogue warp); 8..15 release time
+// of each epilogue warp.
+#ifndef HDQT_TL_Q
+#define HDQT_TL_Q 0   // lane quarter of the epilogue warp whose events are recorded
+#endif
+#ifdef HDQT_TIMELINE
+__device__ long long g_timeline[64 * 16];
+#define HDQT_TL(slot, idx)                                                                            \
+  do {                                                                                                \
+    if (blockIdx.x == 0 && (idx) < 64) g_timeline[(idx) * 16 + (slot)] = clock64();                   \
+  } while (0)
+#else
+#define HDQT_TL(slot, idx) do { } while (0)
+#endif
 
 struct GemmParams {
   int64_t M, N, K_pad;
@@ -46,6 +76,7 @@ struct GemmParams {
   int32_t lo, hi;         // accumulator range
   int32_t had_block;
   int32_t flush_every;    // packed mode: accumulator tiles summed in 16-bit lanes before widening
+  int32_t offset_mma;     // packed mode: every clamp-path accumulator tile starts from the constant 2^(b_a-1)
   // merging of provably clamp-free accumulator tiles
   int32_t merge;          // 0 = off, 1 = certificates from the tile norms, 2 = every tile is clamp-free
   int32_t merge_max_uncert_256;  // a CTA merges only if uncertified tiles <= this/256 of all tiles
@@ -109,14 +140,31 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 //
 // mbar_wait: for the two single-thread roles (TMA producer, MMA issuer), whose waits are on the
 // critical path of every K tile: polls without suspending first, then backs off.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int slow_polls = 1 << 20) {
   for (int i = 0; i < (1 << 12); ++i) {
     if (mbar_test_wait(bar, parity)) return true;
   }
-  for (int i = 0; i < (1 << 20); ++i) {
+  for (int i = 0; i < slow_polls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     __nanosleep(512);
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// mbar_wait_suspend: for waits that are usually long (the TMA producer far ahead of the MMAs, the MMA issuer
+// behind a slower epilogue): try_wait parks the thread in hardware until the phase completes or a short time
+// limit passes, so the waiting warp takes no issue slots from the warps of its scheduler that have work.
+__device__ __forceinline__ bool mbar_wait_suspend(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  long long limit_clk = 2000000000ll) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long start = clock64();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - start > limit_clk) break;
   }
   *abort_flag = 1;
   return false;
@@ -127,10 +175,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // polls; kSleepNs is the poll period (short for the per-tile handshake, long for the one wait on the
 // merged accumulator that spans the whole main loop).
 template <int kSleepNs>
-__device__ __forceinline__ bool mbar_wait_yield(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_yield(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                int polls = (kSleepNs >= 512) ? (1 << 21) : (1 << 24)) {
   if (mbar_try_wait(bar, parity)) return true;
-  constexpr int kLimit = (kSleepNs >= 512) ? (1 << 21) : (1 << 24);
-  for (int i = 0; i < kLimit; ++i) {
+  for (int i = 0; i < polls; ++i) {
     __nanosleep(kSleepNs);
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63) == 63 && *abort_flag) return false;
@@ -145,6 +193,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
       : "memory");
+}
+
+template <int kRegs>
+__device__ __forceinline__ void warpgroup_reg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <int kRegs>
+__device__ __forceinline__ void warpgroup_reg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -175,6 +232,17 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
   return d;
 }
 
+// K-major operand tile without swizzle: 8 rows x 16 bytes are contiguous (128 bytes); `lbo` = distance between
+// the two 16-byte K chunks of a 32-byte K slice, `sbo` = distance between 8-row groups.
+__device__ __forceinline__ uint64_t make_smem_desc_plain(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(lbo >> 4) << 16;
+  d |= (uint64_t)(sbo >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+
 #define HDQT_TMEM_LD32(taddr, v)                                                                        \
   asm volatile(                                                                                         \
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                         \
@@ -200,6 +268,25 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
         "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),      \
         "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),      \
         "=r"(v[29]), "=r"(v[30]), "=r"(v[31])                                                           \
+      : "r"(taddr)                                                                                      \
+      : "memory")
+
+#define HDQT_TMEM_LD64_PACK16(taddr, v)                                                                 \
+  asm volatile(                                                                                         \
+      "tcgen05.ld.sync.aligned.32x32b.x64.pack::16b.b32 "                                               \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                         \
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "                \
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "                \
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"         \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),        \
+        "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),      \
+        "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),      \
+        "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]),      \
+        "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]), "=r"(v[41]), "=r"(v[42]),      \
+        "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]), "=r"(v[49]),      \
+        "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]),      \
+        "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])       \
       : "r"(taddr)                                                                                      \
       : "memory")
 
@@ -411,34 +498,71 @@ __device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx
   return true;
 }
 
-// 16-bit-lane path: tile sums fit int16, b_a <= 8, r = 0.  TMEM is read with two columns packed per
-// register (low half = even column); c - lo = relu(min(P - lo, hi - lo)) per lane in one instruction;
-// sums stay unsigned 16-bit lanes and are widened through the output buffer every flush_every tiles.
+// 16-bit-lane path: tile sums fit int16, b_a <= 8, r = 0.
+//
+// Every clamp-path accumulator tile starts from the constant o = 2^(b_a-1) (the MMA issuer writes it with one
+// MMA of constant operand tiles before the tile's data MMAs), so TMEM holds y = P + o, and the accumulator
+// quantisation c = clamp(P, -o, o-1) becomes c + o = clamp(y, 0, 2^b_a - 1).  TMEM is read with two columns
+// packed per register (low half = even column).  In range, y has no bit outside 2^b_a - 1, in either half:
+// one OR-reduction over the warp's registers proves that no element of the tile clamps, and the registers are
+// then added to the 16-bit lane sums as they are (one three-input logic operation per two registers and one
+// add per register, instead of a clamp per register).  A tile with an element out of range takes the clamp
+// instruction instead.  The sums stay unsigned 16-bit lanes (no carry can cross) and are widened through the
+// output buffer every flush_every tiles; o times the tile count is subtracted when they are unpacked.
+//
+// The logic operations and adds are inline PTX on purpose: written in C++, the compiler pairs the 32-bit adds
+// into two-element vector operations that cost two instructions each (measured: 3x the time).  Being volatile,
+// they also stay behind the tcgen05.wait::ld that makes the registers valid.
+__device__ __forceinline__ void packed_accumulate(uint32_t (&S)[EPI_COLS / 2], uint32_t (&v)[EPI_COLS / 2],
+                                                  uint32_t rng2) {
+  uint32_t any0 = 0u, any1 = 0u, any2 = 0u, any3 = 0u;    // four independent chains
+#pragma unroll
+  for (int i = 0; i < EPI_COLS / 2; i += 8) {
+    asm volatile("lop3.b32 %0, %0, %1, %2, 0xFE;" : "+r"(any0) : "r"(v[i]), "r"(v[i + 1]));
+    asm volatile("lop3.b32 %0, %0, %1, %2, 0xFE;" : "+r"(any1) : "r"(v[i + 2]), "r"(v[i + 3]));
+    asm volatile("lop3.b32 %0, %0, %1, %2, 0xFE;" : "+r"(any2) : "r"(v[i + 4]), "r"(v[i + 5]));
+    asm volatile("lop3.b32 %0, %0, %1, %2, 0xFE;" : "+r"(any3) : "r"(v[i + 6]), "r"(v[i + 7]));
+  }
+#pragma unroll
+  for (int i = 0; i < EPI_COLS / 2; ++i) asm volatile("add.u32 %0, %0, %1;" : "+r"(S[i]) : "r"(v[i]));
+  // Rare: some element of the warp's tile is out of range.  The plain add above may then have carried
+  // between the two lanes of a register; taking the added value out again and putting the clamped one in is
+  // exact all the same (32-bit wrap-around arithmetic).  Written as a loop over an opaque count (0 or 1) so
+  // that the compiler emits a real, warp-uniform branch instead of predicating the clamps into the common path.
+  int redo = __any_sync(0xFFFFFFFFu, (((any0 | any1) | (any2 | any3)) & ~rng2) != 0u) ? 1 : 0;
+  asm volatile("" : "+r"(redo));
+#pragma unroll 1
+  for (int rep = 0; rep < redo; ++rep) {
+#pragma unroll
+    for (int i = 0; i < EPI_COLS / 2; ++i) S[i] += __viaddmin_s16x2_relu(v[i], 0u, rng2) - v[i];
+  }
+}
+
 __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
   uint32_t S[EPI_COLS / 2];
 #pragma unroll
   for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
-  const uint32_t off = (uint32_t)(-p.lo);                    // c - lo lies in [0, hi - lo]
-  const uint32_t off2 = off | (off << 16);
+  const uint32_t off = (uint32_t)(-p.lo);                    // c + off lies in [0, hi - lo]
   const uint32_t rng2 = (uint32_t)(p.hi - p.lo) | ((uint32_t)(p.hi - p.lo) << 16);
   int n_in_S = 0;
   bool parked = false;   // int32 partial sums are parked in the output buffer
-  // Half of the warp's columns at a time through one load buffer; the other epilogue warp of the
-  // scheduler covers the load latency.
+  // One load of the warp's whole row segment (128 columns in 64 registers) per tile; the accumulator goes
+  // back to the MMA issuer as soon as the load has landed, before any arithmetic.  (Arithmetic of a warp does
+  // not overlap its own TMEM load in flight - measured: it gets slower -, so the load is not split or
+  // prefetched; the other epilogue warp of the scheduler fills the load's latency.)
   for (int ci = 0; ci < job.n_clamp_tiles; ++ci) {
     const int buf = job.merging ? 1 : (ci & 1);
-    if (!mbar_wait(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
+    if (!mbar_wait_suspend(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
     tc_fence_after();
-    uint32_t v[EPI_COLS / 4];
-    HDQT_LD_HALF_PACK(e.lane_addr + buf * BN, v);
-    HDQT_WAIT_HALF(v);
-#pragma unroll
-    for (int i = 0; i < EPI_COLS / 4; ++i) S[i] += __viaddmin_s16x2_relu(v[i], off2, rng2);
-    HDQT_LD_HALF_PACK(e.lane_addr + buf * BN + EPI_COLS / 2, v);
-    HDQT_WAIT_HALF(v);                                                 // the buffer is free
+    if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(2, ci);
+    uint32_t v[EPI_COLS / 2];
+    HDQT_TMEM_LD64_PACK16(e.lane_addr + buf * BN, v);
+    tmem_ld_wait();
     release_accumulator(e, buf, drains);
-#pragma unroll
-    for (int i = 0; i < EPI_COLS / 4; ++i) S[EPI_COLS / 4 + i] += __viaddmin_s16x2_relu(v[i], off2, rng2);
+    if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(4, ci);
+    if (e.lane == 0) HDQT_TL(8 + e.grp * 4 + e.q, ci);      // release time of every epilogue warp
+    packed_accumulate(S, v, rng2);
+    if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(5, ci);
     if (++n_in_S == p.flush_every && ci + 1 < job.n_clamp_tiles) {
       // widen: park int32 partial sums in the output buffer
       const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;

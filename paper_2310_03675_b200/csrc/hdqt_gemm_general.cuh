@@ -14,8 +14,9 @@ namespace {
 // per-block fixed costs (TMEM allocation, barrier set-up, pipeline fill) are paid once.
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer, 2 = certificate builder (clamp-free tile bitmask of the
-// next block, from the tile norms), 3..10 = epilogue (TMEM lane quarter = warp % 4, 128 columns each;
-// 11 warps leave each thread 168 registers: the sums of 128 columns plus a load buffer fit without spills).
+// next block, from the tile norms), 3 = spare (completes the control warp group), 4..11 = epilogue (TMEM lane
+// quarter = warp % 4, 128 columns each).  The control warp group hands most of its registers to the two
+// epilogue warp groups (setmaxnreg), which hold the sums of 128 columns plus two TMEM load buffers.
 //
 // kPacked: the per-tile sums fit 16 bits and b_a <= 8, r = 0: TMEM is read with two columns packed
 //          per register, clamp and add work on 16-bit lane pairs (half the ALU work per element).
@@ -105,6 +106,18 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (p.offset_mma) {
+    // Constant operand tiles of the offset MMA: every 16-byte K chunk of the A tile holds o/2 in its first
+    // byte and zeros, every byte of the B tile is 1, so that a 32-byte K slice of any row pair multiplies to
+    // o = 2^(b_a-1), wherever the 8-row groups and K chunks of the descriptor fall inside the tiles.
+    const uint32_t half_off = (uint32_t)(-(p.lo / 2));
+    uint4* ca = reinterpret_cast<uint4*>(smem_al + OFFS_A_OFF);
+    uint4* cb = reinterpret_cast<uint4*>(smem_al + OFFS_B_OFF);
+    for (int i = threadIdx.x; i < OFFS_A_BYTES / 16; i += GEMM_THREADS) ca[i] = make_uint4(half_off, 0u, 0u, 0u);
+    for (int i = threadIdx.x; i < OFFS_B_BYTES / 16; i += GEMM_THREADS)
+      cb[i] = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads them through the async proxy
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -117,6 +130,8 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
            (p.merge == 1 && (int64_t)n_uncert * 256 <= (int64_t)p.merge_max_uncert_256 * num_acc);
   };
 
+  if (warp < NUM_CTRL_WARPS) {
+  warpgroup_reg_dec<CTRL_REGS>();
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
@@ -128,7 +143,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         for (int kb = 0; kb < num_kblocks; ++kb, ++it) {
           const uint32_t s = it % STAGES;
           const uint32_t par = ((it / STAGES) & 1u) ^ 1u;
-          if (!mbar_wait(bar_empty + 8 * s, par, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_suspend(bar_empty + 8 * s, par, abort_flag)) { ok = false; break; }
           mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
           const uint32_t a_dst = smem_base + s * STAGE_BYTES;
           tma_load_2d(a_dst, &map_a, kb * BKB, tile_m * BM, bar_full + 8 * s);
@@ -202,6 +217,9 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       // the next stage's barrier polled ahead; only stages with clamp tiles take the per-tile code.
       const uint64_t desc_a0 = make_smem_desc(smem_base);
       const uint64_t desc_b0 = make_smem_desc(smem_base + A_STAGE);
+      const uint64_t desc_offs_a = make_smem_desc_plain(smem_base + OFFS_A_OFF, 128u, 256u);
+      const uint64_t desc_offs_b = make_smem_desc_plain(smem_base + OFFS_B_OFF, 128u, 256u);
+      const uint32_t offset_mma = (uint32_t)p.offset_mma;
       uint32_t s = 0;            // smem stage
       uint32_t full_par = 0;     // parity of the stage's next "full" phase
       uint32_t fills[2] = {0u, 0u};   // how many times each TMEM accumulator has been handed to the epilogue
@@ -237,7 +255,28 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           uint32_t nib = 0;
           if (p.merge == 2) nib = 0xFu;
           else if (nibble_ok) nib = (cert_mask[kb >> 3] >> ((kb & 7) * 4)) & 0xFu;
-          if (nib == 0xFu && kt0 + 4 <= tiles32) {
+          if (!merging && tpa == 1 && offset_mma) {
+            // Every tile of this block takes the clamp path of the 16-bit-lane epilogue: a short, branch-free
+            // sequence per tile.  (This thread shares its scheduler with two epilogue warps; every instruction
+            // it spends between two tiles is taken from them, and they are the slowest of the eight.  Issuing
+            // the odd tiles from a second thread on another scheduler was tried: the lag moved to that
+            // scheduler's warps and the tile rate stayed the same.)
+            const int nsub = min(tiles32 - kt0, 4);
+            for (int sub = 0; sub < nsub; ++sub) {
+              const uint32_t b = (uint32_t)clamp_idx & 1u;
+              if (!mbar_wait_suspend(bar_tempty + 8 * b, (fills[b] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              HDQT_TL(0, clamp_idx);
+              const uint32_t d = tmem_base + b * BN;
+              tc_mma_i8(d, desc_offs_a, desc_offs_b, 0u);
+              tc_mma_i8(d, desc_a + (uint64_t)(2 * sub), desc_b + (uint64_t)(2 * sub), 1u);
+              HDQT_TL(1, clamp_idx);
+              tc_commit(bar_tfull + 8 * b);
+              ++fills[b];
+              ++clamp_idx;
+            }
+            if (!ok) break;
+          } else if (nib == 0xFu && kt0 + 4 <= tiles32) {
             if (!merged_started) {
               // the merged accumulator (buffer 0) must have been drained by the previous user
               if (!mbar_wait(bar_tempty, (fills[0] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -261,13 +300,16 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 // merged tiles accumulate in buffer 0; clamp tiles use buffer 1 when merging, else 0 / 1
                 cur_buf = cert ? 0 : (merging ? 1 : (clamp_idx & 1));
                 if (!cert || !merged_started) {
-                  if (!mbar_wait(bar_tempty + 8 * cur_buf, (fills[cur_buf] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                  if (!mbar_wait_suspend(bar_tempty + 8 * cur_buf, (fills[cur_buf] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                   tc_fence_after();
                 }
                 d_tmem = tmem_base + cur_buf * BN;
+                if (!cert) HDQT_TL(0, clamp_idx);
+                // a clamp-path tile of the 16-bit-lane epilogue starts from the constant 2^(b_a-1)
+                if (!cert && offset_mma) tc_mma_i8(d_tmem, desc_offs_a, desc_offs_b, 0u);
               }
               uint32_t sub2 = (uint32_t)(2 * (kt - kt0));
-              uint32_t accumulate = cert ? merged_started : (uint32_t)(j != 0);
+              uint32_t accumulate = cert ? merged_started : ((uint32_t)(j != 0) | offset_mma);
               tc_mma_i8(d_tmem, desc_a + sub2, desc_b + sub2, accumulate);
               if (tpa >= 4) {
                 // long accumulator tiles: the rest of this stage's K tiles that belong to the same
@@ -283,6 +325,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
               if (cert) merged_started = 1u;
               if (++j == tpa || kt == tiles32 - 1) {
                 if (!cert) {
+                  HDQT_TL(1, clamp_idx);
                   tc_commit(bar_tfull + 8 * cur_buf);
                   ++fills[cur_buf];
                   ++clamp_idx;
@@ -313,17 +356,19 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (p.merge == 1) mbar_arrive(bar_iempty + 8 * slot);
       }
     }
+  }
   } else {
     // ------------------------------ epilogue warps ----------------------------
+    warpgroup_reg_inc<EPI_REGS>();
     EpiCtx e;
     e.q = warp & 3;                     // TMEM lane quarter this warp may read
-    e.grp = (warp - 3) >> 2;            // which EPI_COLS columns of the accumulator
+    e.grp = (warp - NUM_CTRL_WARPS) >> 2;   // which EPI_COLS columns of the accumulator
     e.lane = lane;
     e.lane_addr = tmem_base + ((uint32_t)(e.q * 32) << 16) + (uint32_t)(e.grp * EPI_COLS);
     e.bar_tfull = bar_tfull;
     e.bar_tempty = bar_tempty;
     e.abort_flag = abort_flag;
-    e.box = reinterpret_cast<float*>(smem_al + OUT_STAGE_OFF + (warp - 3) * OUT_STAGE_WARP);
+    e.box = reinterpret_cast<float*>(smem_al + OUT_STAGE_OFF + (warp - NUM_CTRL_WARPS) * OUT_STAGE_WARP);
     uint32_t drains[2] = {0u, 0u};      // how many times this warp has drained each accumulator
     int ti = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++ti) {

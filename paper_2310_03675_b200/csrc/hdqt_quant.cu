@@ -13,6 +13,12 @@
 // Both are HBM-bound streaming kernels: 4 B/element read (+1 B/element written when
 // quantizing).  Butterfly order is ascending stride, every add/sub is a single fp32 rounding,
 // so the transformed values - and hence the codes - are bit-identical for both layouts.
+//
+// One launch serves up to two operands (the two operands of a GEMM): thread blocks
+// [first_block, first_block + num_blocks) of the grid belong to operand i.  The calibration
+// launch leaves one partial maximum per thread block; every block of the quantize launch
+// reduces those (a few hundred values) itself, so no memset, atomic or extra launch sits
+// between the two passes.
 #include <mutex>
 
 #include "hdqt_common.cuh"
@@ -113,26 +119,42 @@ __device__ __forceinline__ void load8_kc(const float* __restrict__ row, int64_t 
 }
 
 // ---- quantizer --------------------------------------------------------------------------
+// Codes are produced with the offset 2^(bits-1) added (so that they are unsigned and one
+// min-with-relu instruction clamps both sides), packed four to a word, and the offset is taken out
+// of all four bytes at once: (w + addc) ^ 0x80808080 with addc = (0x80 - offset) in every byte
+// (no byte can carry into its neighbour).
 
 struct QuantParams {
   float m;
-  int lo, hi;
   int mode;          // hdqt_round_t
+  int rng;           // 2^bits - 1: the largest offset code
+  int nearest_bias;  // offset - bit pattern of the fp32 rounding constant
+  int sr_bias;       // (offset << 16) - bit pattern of 192.0f
+  int off16;         // offset << 16
+  uint32_t addc;
   bool sr_magic;     // |v| < 64 guaranteed: fixed-point conversion through the fp32 adder
+  bool zero_all;     // degenerate scale (all-zero or non-finite tensor): every code is 0
   uint32_t tag;
   const PhiloxKeys* keys;   // the launch's round keys (a kernel parameter)
 };
 
-// codes of 8 consecutive elements; `g` = (linear index of the first element) / 8
-__device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams& p, uint64_t g,
-                                          int (&c)[8]) {
+__device__ __forceinline__ uint32_t pack4_offset(const int (&t)[8], int base, uint32_t addc) {
+  const uint32_t w = (uint32_t)t[base] | ((uint32_t)t[base + 1] << 8) | ((uint32_t)t[base + 2] << 16) |
+                     ((uint32_t)t[base + 3] << 24);
+  return (w + addc) ^ 0x80808080u;
+}
+
+// codes of 8 consecutive elements as two packed words; `g` = (linear index of the first element) / 8
+__device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams& p, uint64_t g, uint32_t& w0,
+                                          uint32_t& w1) {
+  int t[8];
   if (p.mode == HDQT_ROUND_NEAREST) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float v = __fmul_rn(x[i], p.m);
-      // rint through the fp32 adder: exact for |v| < 2^22
-      const int q = __float_as_int(__fadd_rn(v, 12582912.0f)) - 0x4B400000;
-      c[i] = min(max(q, p.lo), p.hi);
+      // rint through the fp32 adder (exact for |v| < 2^22), plus the code offset
+      const int q = __float_as_int(__fadd_rn(v, 12582912.0f)) + p.nearest_bias;
+      t[i] = __vimin_s32_relu(q, p.rng);
     }
   } else {
     const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, 0u, *p.keys);
@@ -141,41 +163,82 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams
       const float v = __fmul_rn(x[i], p.m);
       const uint32_t word = rnd.w[i >> 1];
       const int u16 = (i & 1) ? (int)(word >> 16) : (int)(word & 0xFFFFu);
-      int v_fx;  // rint(v * 2^16), a Q.16 fixed-point integer
+      int s;  // rint(v * 2^16) + u16 + (offset << 16), a Q.16 fixed-point integer
       if (p.sr_magic) {
         // for v in [-64, 64): v + 192 lies in [128, 256) where one ulp is 2^-16
-        v_fx = __float_as_int(__fadd_rn(v, 192.0f)) - 0x43400000;
+        s = __float_as_int(__fadd_rn(v, 192.0f)) + u16 + p.sr_bias;
       } else {
-        v_fx = __float2int_rn(__fmul_rn(v, 65536.0f));
+        s = __float2int_rn(__fmul_rn(v, 65536.0f)) + u16 + p.off16;
       }
-      const int q = (v_fx + u16) >> 16;  // floor((v_fx + u16) / 2^16)
-      c[i] = min(max(q, p.lo), p.hi);
+      t[i] = __vimin_s32_relu(s >> 16, p.rng);   // floor((v_fx + u16) / 2^16) + offset, clamped
     }
   }
-}
-
-__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
-  return (uint32_t)(a & 0xFF) | ((uint32_t)(b & 0xFF) << 8) | ((uint32_t)(c & 0xFF) << 16) |
-         ((uint32_t)(d & 0xFF) << 24);
+  w0 = pack4_offset(t, 0, p.addc);
+  w1 = pack4_offset(t, 4, p.addc);
+  if (p.zero_all) { w0 = 0u; w1 = 0u; }
 }
 
 __device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bits, float clip, int mode,
                                                    const PhiloxKeys* keys, uint32_t tag) {
   QuantParams p;
+  const int off = 1 << (bits - 1);
   p.m = qs.m;
-  p.lo = -(1 << (bits - 1));
-  p.hi = (1 << (bits - 1)) - 1;
   p.mode = mode;
-  p.sr_magic = ((float)(1 << (bits - 1)) <= 32.0f * clip);  // |v| <= 32 (1 + eps)
+  p.rng = (1 << bits) - 1;
+  p.nearest_bias = off - 0x4B400000;
+  p.sr_bias = (off << 16) - 0x43400000;
+  p.off16 = off << 16;
+  p.addc = (uint32_t)(0x80 - off) * 0x01010101u;
+  p.sr_magic = ((float)off <= 32.0f * clip);  // |v| <= 32 (1 + eps)
+  p.zero_all = qs.zero || qs.bad;
   p.keys = keys;
   p.tag = tag;
   return p;
 }
 
+// ---- one operand of a (batched) launch ------------------------------------------------------
+
+constexpr int kMaxOps = 2;
+
+struct QuantOp {
+  const float* src;
+  int64_t rows, K, K_pad;
+  int64_t ld;               // row stride (K contiguous) or K stride (K strided)
+  float clip;
+  int32_t mode;
+  uint32_t tag;
+  int32_t vec;              // K contiguous: 128-bit loads allowed
+  int32_t seg_log2;         // K contiguous, blocked mapping: log2 of the K segment a thread block covers
+  const float* amax_in;     // quantize: supplied maximum, or nullptr = reduce `partials`
+  uint32_t* partials;       // calibration: one partial maximum (bit pattern) per thread block of this operand
+  int32_t n_partials;
+  float* amax_atomic;       // calibration through the public call: atomic maximum into one float instead
+  float* amax_slot;         // quantize: where the maximum that was used is published (may be null)
+  int8_t* codes;
+  float* step_out;
+  int32_t* tile_norms;
+  int32_t first_block, num_blocks;
+};
+
+struct QuantBatch {
+  QuantOp op[kMaxOps];
+  int32_t n_ops;
+  int32_t had_block;
+  int32_t bits;
+};
+
+// which operand this thread block works on, and its block index within that operand
+__device__ __forceinline__ const QuantOp& my_operand(const QuantBatch& b, int& local_block) {
+  const int second = (b.n_ops > 1 && (int)blockIdx.x >= b.op[1].first_block) ? 1 : 0;
+  local_block = (int)blockIdx.x - b.op[second].first_block;
+  return b.op[second];
+}
+
 // ---- block-wide max -----------------------------------------------------------------------
 
-__device__ __forceinline__ void block_absmax_commit(uint32_t mx, float* amax_out, int32_t* dev_status) {
+__device__ __forceinline__ uint32_t block_max_u32(uint32_t mx) {
   __shared__ uint32_t smax[kThreads / 32];
+  __shared__ uint32_t sres;
   mx = __reduce_max_sync(0xFFFFFFFFu, mx);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (lane == 0) smax[warp] = mx;
@@ -183,18 +246,48 @@ __device__ __forceinline__ void block_absmax_commit(uint32_t mx, float* amax_out
   if (warp == 0) {
     uint32_t v = (lane < kThreads / 32) ? smax[lane] : 0u;
     v = __reduce_max_sync(0xFFFFFFFFu, v);
-    if (lane == 0) {
-      // non-negative floats order like their bit patterns
-      atomicMax(reinterpret_cast<uint32_t*>(amax_out), v);
-      if (v >= 0x7F800000u) report_status(dev_status, HDQT_ERR_NONFINITE);
-    }
+    if (lane == 0) sres = v;
+  }
+  __syncthreads();
+  return sres;
+}
+
+__device__ __forceinline__ void commit_partial_max(const QuantOp& op, int local_block, uint32_t mx,
+                                                   int32_t* dev_status) {
+  const uint32_t v = block_max_u32(mx);
+  if (threadIdx.x == 0) {
+    // non-negative floats order like their bit patterns
+    if (op.amax_atomic != nullptr) atomicMax(reinterpret_cast<uint32_t*>(op.amax_atomic), v);
+    else op.partials[local_block] = v;
+    if (v >= 0x7F800000u) report_status(dev_status, HDQT_ERR_NONFINITE);
   }
 }
 
+// The calibration maximum a quantize block works with: the supplied one, or the maximum of the partial
+// maxima the calibration launch left behind.  Block 0 of the operand publishes scale and maximum.
+__device__ __forceinline__ QuantScale resolve_scale(const QuantOp& op, int local_block, int bits,
+                                                    int32_t* dev_status) {
+  float amax;
+  if (op.amax_in != nullptr) {
+    amax = __ldg(op.amax_in);
+  } else {
+    uint32_t mx = 0u;
+    for (int i = threadIdx.x; i < op.n_partials; i += kThreads) mx = max(mx, __ldcg(op.partials + i));
+    amax = __uint_as_float(block_max_u32(mx));
+  }
+  const QuantScale qs = make_quant_scale(amax, op.clip, bits);
+  if (local_block == 0 && threadIdx.x == 0) {
+    *op.step_out = qs.step;
+    if (op.amax_slot != nullptr && op.amax_in == nullptr) *op.amax_slot = amax;
+    if (qs.bad) report_status(dev_status, HDQT_ERR_NONFINITE);
+  }
+  return qs;
+}
+
 // ---- K-contiguous kernels -------------------------------------------------------------------
-// A thread block walks the tensor in slabs of kUnroll*kThreads chunks (a chunk = 8 consecutive k of one
-// row); every thread first issues the loads of its kUnroll chunks, then transforms them, so that
-// kUnroll*32 bytes per thread are in flight.
+// "linear" mapping: a thread block walks the tensor in slabs of kUnroll*kThreads chunks (a chunk = 8
+// consecutive k of one row); every thread first issues the loads of its kUnroll chunks, then transforms
+// them, so that kUnroll*32 bytes per thread are in flight.
 
 constexpr int kUnrollAbsmax = 4;
 constexpr int kUnrollQuant = 2;
@@ -217,16 +310,21 @@ __device__ __forceinline__ void chunk_to_row_k(const ChunkMap& m, int64_t c, int
 }
 
 __global__ void __launch_bounds__(kThreads)
-absmax_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_row, int64_t K_pad,
-                 int had_block, bool vec, float* amax_out, int32_t* dev_status) {
-  const int64_t chunks_per_row = K_pad >> 3;
-  const int64_t total = rows * chunks_per_row;
+absmax_kc_kernel(const __grid_constant__ QuantBatch b, int32_t* dev_status) {
+  int local_block;
+  const QuantOp& op = my_operand(b, local_block);
+  const float* __restrict__ src = op.src;
+  const int64_t K = op.K, ld_row = op.ld;
+  const bool vec = op.vec != 0;
+  const int had_block = b.had_block;
+  const int64_t chunks_per_row = op.K_pad >> 3;
+  const int64_t total = op.rows * chunks_per_row;
   const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
-  const bool dense = (K == K_pad) && (ld_row == K);
+  const bool dense = (K == op.K_pad) && (ld_row == K);
   const int lane = threadIdx.x & 31;
   uint32_t mx = 0u;
-  for (int64_t base = (int64_t)blockIdx.x * (kThreads * kUnrollAbsmax); base < total;
-       base += (int64_t)gridDim.x * (kThreads * kUnrollAbsmax)) {
+  for (int64_t base = (int64_t)local_block * (kThreads * kUnrollAbsmax); base < total;
+       base += (int64_t)op.num_blocks * (kThreads * kUnrollAbsmax)) {
     float x[kUnrollAbsmax][8];
 #pragma unroll
     for (int u = 0; u < kUnrollAbsmax; ++u) {
@@ -252,34 +350,35 @@ absmax_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t
       for (int i = 0; i < 8; ++i) mx = max(mx, abs_bits(x[u][i]));
     }
   }
-  block_absmax_commit(mx, amax_out, dev_status);
+  commit_partial_max(op, local_block, mx, dev_status);
 }
 
+// quantize, linear mapping (no tile norms)
 __global__ void __launch_bounds__(kThreads)
-quantize_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_row, int64_t K_pad,
-                   int had_block, bool vec, int bits, float clip, int mode,
-                   const __grid_constant__ PhiloxKeys keys, uint32_t tag,
-                   const float* __restrict__ amax_ptr, int8_t* __restrict__ codes, float* step_out,
-                   uint16_t* __restrict__ row_norms, int32_t* dev_status) {
-  const QuantScale qs = make_quant_scale(__ldg(amax_ptr), clip, bits);
-  const QuantParams p = make_params(qs, bits, clip, mode, &keys, tag);
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    *step_out = qs.step;
-    if (qs.bad) report_status(dev_status, HDQT_ERR_NONFINITE);
-  }
-  const int64_t chunks_per_row = K_pad >> 3;
-  const int64_t total = rows * chunks_per_row;
+quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__ PhiloxKeys keys,
+                   int32_t* dev_status) {
+  int local_block;
+  const QuantOp& op = my_operand(b, local_block);
+  const QuantScale qs = resolve_scale(op, local_block, b.bits, dev_status);
+  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag);
+  const float* __restrict__ src = op.src;
+  int8_t* __restrict__ codes = op.codes;
+  const int64_t K = op.K, ld_row = op.ld;
+  const bool vec = op.vec != 0;
+  const int had_block = b.had_block;
+  const int64_t chunks_per_row = op.K_pad >> 3;
+  const int64_t total = op.rows * chunks_per_row;
   const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
-  const bool dense = (K == K_pad) && (ld_row == K);
+  const bool dense = (K == op.K_pad) && (ld_row == K);
   const int lane = threadIdx.x & 31;
-  for (int64_t base = (int64_t)blockIdx.x * (kThreads * kUnrollQuant); base < total;
-       base += (int64_t)gridDim.x * (kThreads * kUnrollQuant)) {
+  for (int64_t base = (int64_t)local_block * (kThreads * kUnrollQuant); base < total;
+       base += (int64_t)op.num_blocks * (kThreads * kUnrollQuant)) {
     float x[kUnrollQuant][8];
 #pragma unroll
     for (int u = 0; u < kUnrollQuant; ++u) {
       const int64_t c = base + u * kThreads + threadIdx.x;
       if (c < total) {
-        if (dense) {   // rows are back to back and unpadded: chunk c starts at element 8c
+        if (dense) {
           load8_kc(src, c << 3, total << 3, vec, x[u]);
         } else {
           int64_t r, k0;
@@ -294,55 +393,92 @@ quantize_kc_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64
 #pragma unroll
     for (int u = 0; u < kUnrollQuant; ++u) {
       const int64_t c = base + u * kThreads + threadIdx.x;
-      const bool valid = c < total;
       fwht8_regs(x[u], had_block);
       fwht8_lanes(x[u], had_block, lane);
-      int q[8];
-      quantize8(x[u], p, (uint64_t)c, q);  // linear index of the chunk's first element is 8*c
-      // codes are dense [rows, K_pad]: chunk c is bytes [8c, 8c+8) and tile c/4 of the row-norm array
       uint2 out;
-      out.x = pack4(q[0], q[1], q[2], q[3]);
-      out.y = pack4(q[4], q[5], q[6], q[7]);
-      if (row_norms != nullptr) {
-        int ss = __dp4a((int)out.x, (int)out.x, 0);
-        ss = __dp4a((int)out.y, (int)out.y, ss);
-        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
-        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
-        if (valid && (lane & 3) == 0) row_norms[c >> 2] = (uint16_t)ss;
-      }
-      if (valid) *reinterpret_cast<uint2*>(codes + (c << 3)) = out;
+      quantize8(x[u], p, (uint64_t)c, out.x, out.y);  // linear index of the chunk's first element is 8*c
+      // codes are dense [rows, K_pad]: chunk c is bytes [8c, 8c+8)
+      if (c < total) *reinterpret_cast<uint2*>(codes + (c << 3)) = out;
     }
   }
 }
 
-// max over each block of 128 rows of the per-row tile norms: a thread block covers 64 K tiles of one
-// row block, its 4 thread rows take 32 rows each, shared memory combines them
-__global__ void __launch_bounds__(256)
-block_norms_kernel(const uint16_t* __restrict__ row_norms, int64_t rows, int64_t T,
-                   int32_t* __restrict__ tile_norms) {
-  __shared__ int s_part[4][64];
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-  const int64_t t = (int64_t)blockIdx.x * 64 + tx;
-  const int64_t rb = blockIdx.y;
-  const int64_t r0 = rb * 128 + ty * 32;
-  int mx = 0;
-  if (t < T) {
-    const uint16_t* p = row_norms + r0 * T + t;
-    if (r0 + 32 <= rows) {
-      // whole group in range: no per-row test, so the 32 independent loads can all be in flight
-      int v[32];
+// quantize, blocked mapping, with the tile norms: a work item is 128 rows x one K segment of 2^seg_log2
+// elements (32..256), so that the maximum over the 128 rows of every tile's sum(code^2) is formed inside
+// the thread block and written once.  A row's segment is covered by seg/8 neighbouring lanes; a warp
+// covers 32/(seg/8) rows per pass, the block's 8 warps cover consecutive rows.
+__global__ void __launch_bounds__(kThreads)
+quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__ PhiloxKeys keys,
+                         int32_t* dev_status) {
+  __shared__ int s_norm[kThreads / 32][32];
+  int local_block;
+  const QuantOp& op = my_operand(b, local_block);
+  const QuantScale qs = resolve_scale(op, local_block, b.bits, dev_status);
+  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag);
+  const float* __restrict__ src = op.src;
+  int8_t* __restrict__ codes = op.codes;
+  const int64_t K = op.K, K_pad = op.K_pad, ld_row = op.ld, rows = op.rows;
+  const bool vec = op.vec != 0;
+  const int had_block = b.had_block;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int lpr_log2 = op.seg_log2 - 3;          // lanes per row segment
+  const int rpw = 32 >> lpr_log2;                // rows per warp pass
+  const int row_sub = lane >> lpr_log2;
+  const int kc = lane & ((1 << lpr_log2) - 1);
+  const int passes = 16 / rpw;                   // 128 rows / (8 warps x rpw rows)
+  const int64_t nseg = (K_pad + (int64_t(1) << op.seg_log2) - 1) >> op.seg_log2;
+  const int64_t T = K_pad >> 5;
+  const int64_t cpr = K_pad >> 3;                // chunks per code row
+  const int64_t n_items = ((rows + 127) >> 7) * nseg;
+  for (int64_t item = local_block; item < n_items; item += op.num_blocks) {
+    const int64_t rb = item / nseg, kseg = item - rb * nseg;
+    const int64_t k0 = (kseg << op.seg_log2) + (kc << 3);
+    const bool k_ok = k0 < K_pad;
+    int nmax = 0;
+    for (int pass = 0; pass < passes; pass += kUnrollQuant) {
+      float x[kUnrollQuant][8];
+      int64_t r[kUnrollQuant];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = (int)__ldg(p + i * T);
+      for (int u = 0; u < kUnrollQuant; ++u) {
+        r[u] = (rb << 7) + (int64_t)((pass + u) * 8 + warp) * rpw + row_sub;
+        if (k_ok && pass + u < passes && r[u] < rows) {
+          load8_kc(src + r[u] * ld_row, k0, K, vec, x[u]);
+        } else {
+          r[u] = -1;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) mx = max(mx, v[i]);
-    } else {
-      for (int i = 0; i < 32 && r0 + i < rows; ++i) mx = max(mx, (int)__ldg(p + i * T));
+          for (int i = 0; i < 8; ++i) x[u][i] = 0.0f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kUnrollQuant; ++u) {
+        fwht8_regs(x[u], had_block);
+        fwht8_lanes(x[u], had_block, lane);
+        const bool valid = r[u] >= 0;
+        const uint64_t g = valid ? (uint64_t)r[u] * (uint64_t)cpr + (uint64_t)(k0 >> 3) : 0u;
+        uint2 out;
+        quantize8(x[u], p, g, out.x, out.y);
+        int ss = __dp4a((int)out.x, (int)out.x, 0);
+        ss = __dp4a((int)out.y, (int)out.y, ss);
+        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+        if (valid) {
+          nmax = max(nmax, ss);
+          *reinterpret_cast<uint2*>(codes + r[u] * K_pad + k0) = out;
+        }
+      }
     }
-  }
-  s_part[ty][tx] = mx;
-  __syncthreads();
-  if (ty == 0 && t < T) {
-    tile_norms[rb * T + t] = max(max(s_part[0][tx], s_part[1][tx]), max(s_part[2][tx], s_part[3][tx]));
+    s_norm[warp][lane] = nmax;
+    __syncthreads();
+    if ((int)threadIdx.x < (1 << (op.seg_log2 - 5))) {
+      const int64_t t = (kseg << (op.seg_log2 - 5)) + threadIdx.x;
+      if (t < T) {
+        int mx = 0;
+        for (int w = 0; w < kThreads / 32; ++w)
+          for (int rs = 0; rs < rpw; ++rs) mx = max(mx, s_norm[w][(rs << lpr_log2) + 4 * (int)threadIdx.x]);
+        op.tile_norms[rb * T + t] = mx;
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -363,13 +499,17 @@ __device__ __forceinline__ void load32_ks(const float* __restrict__ src, int64_t
 }
 
 __global__ void __launch_bounds__(kThreads, 3)
-absmax_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_k, int64_t K_pad,
-                 int had_block, float* amax_out, int32_t* dev_status) {
+absmax_ks_kernel(const __grid_constant__ QuantBatch b, int32_t* dev_status) {
+  int local_block;
+  const QuantOp& op = my_operand(b, local_block);
+  const float* __restrict__ src = op.src;
+  const int64_t rows = op.rows, K = op.K, ld_k = op.ld;
+  const int had_block = b.had_block;
   // work item = (32-block of K, group of kThreads rows); the host guarantees that their number fits 31 bits
   const uint32_t row_groups = (uint32_t)((rows + kThreads - 1) / kThreads);
-  const uint32_t items = row_groups * (uint32_t)(K_pad >> 5);
+  const uint32_t items = row_groups * (uint32_t)(op.K_pad >> 5);
   uint32_t mx = 0u;
-  for (uint32_t w = blockIdx.x; w < items; w += gridDim.x) {
+  for (uint32_t w = (uint32_t)local_block; w < items; w += (uint32_t)op.num_blocks) {
     const uint32_t kbu = w / row_groups;
     const int64_t kb = kbu;
     const int64_t r = (int64_t)(w - kbu * row_groups) * kThreads + threadIdx.x;
@@ -381,29 +521,29 @@ absmax_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t
       for (int i = 0; i < 32; ++i) mx = max(mx, abs_bits(x[i]));
     }
   }
-  block_absmax_commit(mx, amax_out, dev_status);
+  commit_partial_max(op, local_block, mx, dev_status);
 }
 
 __global__ void __launch_bounds__(kThreads, 3)
-quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64_t ld_k, int64_t K_pad,
-                   int had_block, int bits, float clip, int mode,
-                   const __grid_constant__ PhiloxKeys keys, uint32_t tag,
-                   const float* __restrict__ amax_ptr, int8_t* __restrict__ codes, float* step_out,
-                   int32_t* __restrict__ tile_norms, int32_t* dev_status) {
+quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__ PhiloxKeys keys,
+                   int32_t* dev_status) {
   __shared__ int s_norm[kThreads / 32];
-  const QuantScale qs = make_quant_scale(__ldg(amax_ptr), clip, bits);
-  const QuantParams p = make_params(qs, bits, clip, mode, &keys, tag);
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    *step_out = qs.step;
-    if (qs.bad) report_status(dev_status, HDQT_ERR_NONFINITE);
-  }
+  int local_block;
+  const QuantOp& op = my_operand(b, local_block);
+  const QuantScale qs = resolve_scale(op, local_block, b.bits, dev_status);
+  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag);
+  const float* __restrict__ src = op.src;
+  int8_t* __restrict__ codes = op.codes;
+  int32_t* __restrict__ tile_norms = op.tile_norms;
+  const int64_t rows = op.rows, K = op.K, K_pad = op.K_pad, ld_k = op.ld;
+  const int had_block = b.had_block;
   // rows are padded to a multiple of the block size so that one thread block never straddles
   // two 32-blocks of K and always covers whole 128-row groups (needed for the tile norms)
   const int64_t T = K_pad >> 5;
   const uint32_t row_groups = (uint32_t)((rows + kThreads - 1) / kThreads);
   const uint32_t items = row_groups * (uint32_t)T;   // the host guarantees that this fits 31 bits
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
+  for (uint32_t item = (uint32_t)local_block; item < items; item += (uint32_t)op.num_blocks) {
     const uint32_t kbu = item / row_groups;     // uniform over the block
     const int64_t kb = kbu;
     const int64_t r_group0 = (int64_t)(item - kbu * row_groups) * kThreads;
@@ -418,12 +558,9 @@ quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         float x8[8];
-        int q[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) x8[i] = x[8 * j + i];
-        quantize8(x8, p, g0 + j, q);
-        w[2 * j] = pack4(q[0], q[1], q[2], q[3]);
-        w[2 * j + 1] = pack4(q[4], q[5], q[6], q[7]);
+        quantize8(x8, p, g0 + j, w[2 * j], w[2 * j + 1]);
         ss = __dp4a((int)w[2 * j], (int)w[2 * j], ss);
         ss = __dp4a((int)w[2 * j + 1], (int)w[2 * j + 1], ss);
       }
@@ -449,74 +586,157 @@ quantize_ks_kernel(const float* __restrict__ src, int64_t rows, int64_t K, int64
   }
 }
 
-int g_sm_count = 0;
+constexpr int kMaxDevices = 64;
+
+int grid_for(int64_t work_items, int per_block, int blocks_per_sm) {
+  const int64_t need = (work_items + per_block - 1) / per_block;
+  const int64_t cap = (int64_t)sm_count() * blocks_per_sm;
+  const int64_t g = need < 1 ? 1 : (need < cap ? need : cap);
+  return (int)(g < kMaxPartials ? g : kMaxPartials);
+}
+
+// K segment of the blocked mapping: the widest of 256/128/64/32 that wastes at most 1/8 of its lanes
+int pick_seg_log2(int64_t K_pad) {
+  for (int s = 8; s > 5; --s) {
+    const int64_t seg = int64_t(1) << s;
+    const int64_t covered = (K_pad + seg - 1) / seg * seg;
+    if (covered * 8 <= K_pad * 9) return s;
+  }
+  return 5;
+}
+
+QuantOp make_op(const QuantOperand& a, int32_t had_block, uint32_t* partials) {
+  QuantOp o;
+  o.src = a.src;
+  o.rows = a.rows;
+  o.K = a.K;
+  o.K_pad = hdqt_padded_k(a.K, had_block);
+  const bool kc = (a.ld_k == 1);
+  o.ld = kc ? a.ld_row : a.ld_k;
+  o.clip = a.clip;
+  o.mode = a.mode;
+  o.tag = a.tag;
+  o.vec = (kc && (a.ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0)) ? 1 : 0;
+  o.seg_log2 = pick_seg_log2(o.K_pad);
+  o.amax_in = a.amax_in;
+  o.partials = partials;
+  o.n_partials = 0;
+  o.amax_atomic = nullptr;
+  o.amax_slot = a.amax_slot;
+  o.codes = a.codes;
+  o.step_out = a.step_out;
+  o.tile_norms = a.tile_norms;
+  o.first_block = 0;
+  o.num_blocks = 0;
+  return o;
+}
 
 }  // namespace
 
 int sm_count() {
-  if (g_sm_count == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
-      n = kNumSMsHint;
-    }
-    g_sm_count = n;
+  static int cache[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return kNumSMsHint;
+  if (cache[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = kNumSMsHint;
+    cache[dev] = n;
   }
-  return g_sm_count;
-}
-
-static int grid_for(int64_t work_items, int per_block, int blocks_per_sm) {
-  const int64_t need = (work_items + per_block - 1) / per_block;
-  const int64_t cap = (int64_t)sm_count() * blocks_per_sm;
-  return (int)(need < 1 ? 1 : (need < cap ? need : cap));
+  return cache[dev];
 }
 
 hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
-                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s,
-                            bool zero_first) {
-  const int64_t K_pad = hdqt_padded_k(K, had_block);
-  if (zero_first && cudaMemsetAsync(amax_out, 0, sizeof(float), s) != cudaSuccess) return HDQT_ERR_CUDA;
+                            int32_t had_block, float* amax_out, int32_t* dev_status, cudaStream_t s) {
+  if (cudaMemsetAsync(amax_out, 0, sizeof(float), s) != cudaSuccess) return HDQT_ERR_CUDA;
+  QuantOperand a{};
+  a.src = src; a.rows = rows; a.K = K; a.ld_row = ld_row; a.ld_k = ld_k;
+  QuantBatch b{};
+  b.n_ops = 1;
+  b.had_block = had_block;
+  b.bits = 4;
+  b.op[0] = make_op(a, had_block, nullptr);
+  b.op[0].amax_atomic = amax_out;
   if (ld_k == 1) {
-    const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
-    const int64_t total = rows * (K_pad >> 3);
-    absmax_kc_kernel<<<grid_for(total, kThreads * kUnrollAbsmax, 4), kThreads, 0, s>>>(
-        src, rows, K, ld_row, K_pad, had_block, vec, amax_out, dev_status);
+    b.op[0].num_blocks = grid_for(rows * (b.op[0].K_pad >> 3), kThreads * kUnrollAbsmax, 4);
+    absmax_kc_kernel<<<b.op[0].num_blocks, kThreads, 0, s>>>(b, dev_status);
   } else {
-    const int64_t items = ((rows + kThreads - 1) / kThreads) * (K_pad >> 5);
+    const int64_t items = ((rows + kThreads - 1) / kThreads) * (b.op[0].K_pad >> 5);
     if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
-    absmax_ks_kernel<<<grid_for(items, 1, 3), kThreads, 0, s>>>(src, rows, K, ld_k, K_pad, had_block, amax_out,
-                                                              dev_status);
+    b.op[0].num_blocks = grid_for(items, 1, 3);
+    absmax_ks_kernel<<<b.op[0].num_blocks, kThreads, 0, s>>>(b, dev_status);
   }
   return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
 }
 
-hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t ld_row, int64_t ld_k,
-                              int32_t had_block, int32_t bits, float clip, int32_t mode, uint64_t seed,
-                              uint32_t tag, const float* amax, int8_t* codes, float* step_out,
-                              int32_t* tile_norms, uint16_t* row_norms_scratch, int32_t* dev_status,
-                              cudaStream_t s) {
-  const int64_t K_pad = hdqt_padded_k(K, had_block);
-  const int64_t T = K_pad >> 5;
-  const PhiloxKeys keys = make_philox_keys(seed);
-  if (ld_k == 1) {
-    const bool vec = (ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
-    const int64_t total = rows * (K_pad >> 3);
-    uint16_t* rn = tile_norms ? row_norms_scratch : nullptr;
-    quantize_kc_kernel<<<grid_for(total, kThreads * kUnrollQuant, 4), kThreads, 0, s>>>(
-        src, rows, K, ld_row, K_pad, had_block, vec, bits, clip, mode, keys, tag, amax, codes, step_out, rn,
-        dev_status);
-    if (tile_norms) {
-      dim3 grid((unsigned)((T + 63) / 64), (unsigned)((rows + 127) / 128));
-      block_norms_kernel<<<grid, 256, 0, s>>>(rn, rows, T, tile_norms);
+hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int32_t had_block, int32_t bits,
+                                        uint64_t seed, uint32_t* partials, int32_t* dev_status, cudaStream_t s) {
+  if (n_ops < 1 || n_ops > kMaxOps) return HDQT_ERR_INVALID_ARG;
+  QuantOp op[kMaxOps];
+  for (int i = 0; i < n_ops; ++i) {
+    op[i] = make_op(ops[i], had_block, partials + (size_t)i * kMaxPartials);
+    if (ops[i].ld_k != 1) {
+      const int64_t items = ((ops[i].rows + kThreads - 1) / kThreads) * (op[i].K_pad >> 5);
+      if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
     }
-  } else {
-    const int64_t items = ((rows + kThreads - 1) / kThreads) * T;
-    if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
-    quantize_ks_kernel<<<grid_for(items, 1, 3), kThreads, 0, s>>>(
-        src, rows, K, ld_k, K_pad, had_block, bits, clip, mode, keys, tag, amax, codes, step_out, tile_norms,
-        dev_status);
   }
-  return cudaGetLastError() == cudaSuccess ? HDQT_OK : HDQT_ERR_CUDA;
+  // ---- calibration pass: operands without a supplied maximum, one launch per memory layout
+  for (int layout = 0; layout < 2; ++layout) {   // 0 = K contiguous, 1 = K strided
+    QuantBatch b{};
+    b.had_block = had_block;
+    b.bits = bits;
+    int grid = 0;
+    for (int i = 0; i < n_ops; ++i) {
+      if ((ops[i].ld_k != 1) != (layout == 1) || ops[i].amax_in != nullptr) continue;
+      int g;
+      if (layout == 0) {
+        g = grid_for(op[i].rows * (op[i].K_pad >> 3), kThreads * kUnrollAbsmax, 4);
+      } else {
+        g = grid_for(((op[i].rows + kThreads - 1) / kThreads) * (op[i].K_pad >> 5), 1, 3);
+      }
+      op[i].n_partials = g;
+      QuantOp& o = b.op[b.n_ops++];
+      o = op[i];
+      o.first_block = grid;
+      o.num_blocks = g;
+      grid += g;
+    }
+    if (b.n_ops == 0) continue;
+    if (layout == 0) absmax_kc_kernel<<<grid, kThreads, 0, s>>>(b, dev_status);
+    else absmax_ks_kernel<<<grid, kThreads, 0, s>>>(b, dev_status);
+    if (cudaGetLastError() != cudaSuccess) return HDQT_ERR_CUDA;
+  }
+  // ---- quantize pass: one launch per kernel variant
+  const PhiloxKeys keys = make_philox_keys(seed);
+  for (int variant = 0; variant < 3; ++variant) {   // 0 = K contiguous, 1 = K contiguous + tile norms, 2 = K strided
+    QuantBatch b{};
+    b.had_block = had_block;
+    b.bits = bits;
+    int grid = 0;
+    for (int i = 0; i < n_ops; ++i) {
+      const int v = (ops[i].ld_k != 1) ? 2 : (ops[i].tile_norms != nullptr ? 1 : 0);
+      if (v != variant) continue;
+      int g;
+      if (variant == 0) {
+        g = grid_for(op[i].rows * (op[i].K_pad >> 3), kThreads * kUnrollQuant, 4);
+      } else if (variant == 1) {
+        const int64_t seg = int64_t(1) << op[i].seg_log2;
+        g = grid_for(((op[i].rows + 127) / 128) * ((op[i].K_pad + seg - 1) / seg), 1, 4);
+      } else {
+        g = grid_for(((op[i].rows + kThreads - 1) / kThreads) * (op[i].K_pad >> 5), 1, 3);
+      }
+      QuantOp& o = b.op[b.n_ops++];
+      o = op[i];
+      o.first_block = grid;
+      o.num_blocks = g;
+      grid += g;
+    }
+    if (b.n_ops == 0) continue;
+    if (variant == 0) quantize_kc_kernel<<<grid, kThreads, 0, s>>>(b, keys, dev_status);
+    else if (variant == 1) quantize_kc_norms_kernel<<<grid, kThreads, 0, s>>>(b, keys, dev_status);
+    else quantize_ks_kernel<<<grid, kThreads, 0, s>>>(b, keys, dev_status);
+    if (cudaGetLastError() != cudaSuccess) return HDQT_ERR_CUDA;
+  }
+  return HDQT_OK;
 }
 
 }  // namespace hdqt
@@ -524,15 +744,14 @@ hdqt_status_t launch_quantize(const float* src, int64_t rows, int64_t K, int64_t
 // ---- allocation-free variant of the transform + quantize call ----------------------------------
 //
 // Scratch for hdqt_quantize_hadamard_static lives in this fixed device array instead of a caller
-// workspace: [0, 256) holds the calibration maximum, the rest holds the per-row tile norms.
+// workspace: the partial maxima that the calibration pass hands to the quantize pass.
 // Every GPU that loads the library carries these HDQT_STATIC_SCRATCH_BYTES until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[HDQT_STATIC_SCRATCH_BYTES];
 
 namespace {
 
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
-void* g_static_scratch_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+void* g_static_scratch_ptr[hdqt::kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
 
 // In host code the name g_static_scratch is only a handle for the runtime, not a device address;
 // the address a kernel can use must be asked for, once per device, with that device current.
@@ -540,7 +759,7 @@ hdqt_status_t static_scratch_for_current_device(unsigned char** out) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return hdqt::cuda_failure(e, "cudaGetDevice(static scratch)");
-  if (dev < 0 || dev >= kMaxDevices) return HDQT_ERR_UNSUPPORTED;
+  if (dev < 0 || dev >= hdqt::kMaxDevices) return HDQT_ERR_UNSUPPORTED;
   std::lock_guard<std::mutex> lock(g_static_mutex);
   if (g_static_scratch_ptr[dev] == nullptr) {
     void* ptr = nullptr;
@@ -568,20 +787,21 @@ extern "C" hdqt_status_t hdqt_quantize_hadamard_static(const float* src, int64_t
   if (!(clip >= 1.0f / 64.0f && clip <= 1.0f)) return HDQT_ERR_INVALID_ARG;
   if (mode != HDQT_ROUND_NEAREST && mode != HDQT_ROUND_STOCHASTIC) return HDQT_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(src) & 3) || (reinterpret_cast<uintptr_t>(codes) & 127)) return HDQT_ERR_ALIGNMENT;
-  // the fixed array bounds the operand: 256 bytes + 2 bytes per (row, 32-wide K tile)
+  // the stated maximum of this entry point: rows * (K_pad / 32) <= HDQT_STATIC_MAX_ROW_TILES
   const int64_t tiles = hdqt_padded_k(K, had_block) / 32;
-  if (rows > (int64_t)(HDQT_STATIC_SCRATCH_BYTES - 256) / 2 / tiles) return HDQT_ERR_STATIC_SCRATCH;
+  if (rows > (int64_t)HDQT_STATIC_MAX_ROW_TILES / tiles) return HDQT_ERR_STATIC_SCRATCH;
 
   unsigned char* scratch = nullptr;
   hdqt_status_t st = static_scratch_for_current_device(&scratch);
   if (st != HDQT_OK) return st;
-  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  float* amax = reinterpret_cast<float*>(scratch);
-  uint16_t* row_norms = reinterpret_cast<uint16_t*>(scratch + 256);
-  // the array keeps whatever the previous call left: launch_absmax zeroes the maximum before it
-  // accumulates into it, and every row-norm entry that is read is written first by this call
-  st = hdqt::launch_absmax(src, rows, K, ld_row, ld_k, had_block, amax, dev_status, s);
-  if (st != HDQT_OK) return st;
-  return hdqt::launch_quantize(src, rows, K, ld_row, ld_k, had_block, bits, clip, mode, seed, tag, amax, codes,
-                               step_out, tile_norms, row_norms, dev_status, s);
+  // the array keeps whatever the previous call left: the calibration pass overwrites every partial
+  // maximum that the quantize pass of this call reads, so nothing needs clearing
+  hdqt::QuantOperand a{};
+  a.src = src; a.rows = rows; a.K = K; a.ld_row = ld_row; a.ld_k = ld_k;
+  a.clip = clip; a.mode = mode; a.tag = tag;
+  a.amax_in = nullptr;
+  a.amax_slot = reinterpret_cast<float*>(scratch);
+  a.codes = codes; a.step_out = step_out; a.tile_norms = tile_norms;
+  return hdqt::launch_calibrate_quantize(&a, 1, had_block, bits, seed, reinterpret_cast<uint32_t*>(scratch + 256),
+                                         dev_status, reinterpret_cast<cudaStream_t>(stream));
 }

@@ -18,13 +18,15 @@ ROUND_NEAREST = 0
 ROUND_STOCHASTIC = 1
 FLAG_NO_MERGE = 1
 
-STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "WORKSPACE", "NONFINITE", "TIMEOUT", "CUDA"]
+STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "WORKSPACE", "NONFINITE", "TIMEOUT", "CUDA",
+                "STATIC_SCRATCH"]
 
 EXPORTED = [
     "hdqt_default_desc", "hdqt_padded_k", "hdqt_status_string", "hdqt_absmax_hadamard",
     "hdqt_quantize_hadamard", "hdqt_quantize_workspace_bytes", "hdqt_gemm_i8_tiled",
     "hdqt_gemm_i8_workspace_bytes", "hdqt_calibrate_acc_shift", "hdqt_gemm_fwd", "hdqt_gemm_dgrad",
     "hdqt_gemm_wgrad", "hdqt_workspace_bytes", "hdqt_workspace_layout", "hdqt_quantize_hadamard_static",
+    "hdqt_selftest_bounded_wait",
 ]
 
 
@@ -50,9 +52,13 @@ def _load() -> C.CDLL:
     if not os.path.exists(path) or _build.needs_rebuild():
         try:
             _build.build()
-        except Exception as e:  # no silent fallback: the product needs its CUDA library
-            if not os.path.exists(path):
-                raise ImportError(f"HDQT CUDA library missing and could not be built: {e}") from e
+        except Exception as e:
+            # No silent fallback: neither to a CPU path nor to a library older than the sources beside it.
+            # A box without the CUDA toolkit may still load a library that was built elsewhere from these
+            # very sources (the build stamps their digest next to it).
+            if not (os.path.exists(path) and _build.stamp_matches_sources()):
+                raise ImportError(f"HDQT CUDA library is missing or older than its sources and could not be "
+                                  f"rebuilt: {e}") from e
     lib = C.CDLL(path)
     i32, i64, u32, u64, f32, vp, sz = C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_float, C.c_void_p, C.c_size_t
     lib.hdqt_default_desc.argtypes = [C.POINTER(GemmDesc), C.c_int]
@@ -76,6 +82,8 @@ def _load() -> C.CDLL:
     lib.hdqt_calibrate_acc_shift.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, sz, vp, vp]
     for name in ("hdqt_gemm_fwd", "hdqt_gemm_dgrad", "hdqt_gemm_wgrad"):
         getattr(lib, name).argtypes = [C.POINTER(GemmDesc), vp, vp, vp, i64, i64, i64, i32, vp, sz, vp, vp]
+    lib.hdqt_selftest_bounded_wait.argtypes = [vp, vp, vp]
+    lib.hdqt_selftest_bounded_wait.restype = C.c_int
     lib.hdqt_workspace_bytes.argtypes = [C.POINTER(GemmDesc), i64, i64, i64]
     lib.hdqt_workspace_bytes.restype = sz
     lib.hdqt_workspace_layout.argtypes = [C.POINTER(GemmDesc), i64, i64, i64, C.POINTER(WsLayout)]
@@ -174,7 +182,8 @@ def quantize_hadamard(src: torch.Tensor, had_block: int = 32, bits: int = 4, cli
     return codes, step, norms
 
 
-STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 + 256
+STATIC_SCRATCH_BYTES = 256 + 4096
+STATIC_MAX_ROW_TILES = 2097152
 
 
 def quantize_hadamard_static(src: torch.Tensor, codes: torch.Tensor, step: torch.Tensor,

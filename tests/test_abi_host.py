@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(hdqt):
 
 def test_status_strings(hdqt):
     seen = set()
-    for code in range(8):
+    for code in range(9):
         s = hdqt.lib.hdqt_status_string(code).decode()
         assert s and s not in seen
         seen.add(s)

@@ -457,3 +457,81 @@ def test_work_split_ragged_shapes_and_unaligned_output(hdqt):
         assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
         assert np.array_equal(out.cpu().numpy(), want_out)
     assert (big[:, 0] == -7.0).all().item() and (big[:, N + 1:] == -7.0).all().item()
+
+
+@pytest.mark.parametrize("in_bits,acc_bits", [(7, 8), (8, 8), (7, 16), (8, 16)])
+def test_merging_with_wide_codes_uses_exact_tile_norms(hdqt, in_bits, acc_bits):
+    """7/8-bit codes: a tile's sum(code^2) exceeds 16 bits, so a truncated norm would certify tiles that clamp.
+    Composite call with merging on (enough output blocks for the norms to be produced) against the oracle."""
+    Nb, D, C = 128 * 8 + 40, 256 * 4 + 24, 192            # dgrad: M = Nb, N = D: 9 x 5 = 45 output blocks
+    G = inputs.gradients(Nb, C, seed=in_bits)
+    G[5, :] *= 40.0                                       # one loud row: most other codes are small, some tiles certify
+    W = inputs.weights(D, C, seed=acc_bits)
+    over = dict(in_bits=in_bits, acc_bits=acc_bits, clip_a=0.25, clip_b=0.25, seed=3)
+    want = O.gemm_dgrad(G, W, O.dgrad_desc(tag_a=2, tag_b=3, **over))
+    status = hdqt.new_status("cuda")
+    out, ws = hdqt.gemm_dgrad(_dev(G), _dev(W), desc=hdqt.default_desc("dgrad", **over), dev_status=status)
+    hdqt.check_device_status(status)
+    assert np.array_equal(ws.codes_a().cpu().numpy(), want["Aq"])
+    assert np.array_equal(ws.codes_b().cpu().numpy(), want["Bq"])
+    assert np.array_equal(out.cpu().numpy(), want["out"])
+
+
+def test_packed_epilogue_limit_with_two_bit_codes(hdqt):
+    """code_bits = 2, acc_tile = 8160: a tile sum reaches 32640, and 32640 + 128 no longer fits the signed
+    16-bit lanes of the packed epilogue, so the 32-bit epilogue must be chosen."""
+    K = 8160
+    A = np.full((40, K), -2, np.int8)
+    B = np.full((24, K), -2, np.int8)
+    one = torch.ones(1, device="cuda")
+    _, S, _ = hdqt.gemm_i8_tiled(_dev(A), _dev(B), one, one, 8, 8160, 0, 32, code_bits=2, want_S=True)
+    assert (S == 127).all().item()                        # +32640 saturates at +127
+    _, S, _ = hdqt.gemm_i8_tiled(_dev(A), _dev(-B), one, one, 8, 8160, 0, 32, code_bits=2, want_S=True)
+    assert (S == -128).all().item()
+
+
+def test_clamp_path_rare_and_frequent_saturation(hdqt):
+    """The 16-bit-lane epilogue adds a register batch unclamped when an OR-reduction proves it in range and
+    clamps it otherwise: operands where no tile, a few tiles, and most tiles leave the 8-bit range, merging off."""
+    rng = np.random.default_rng(123)
+    M, N, K = 260, 520, 32 * 40
+    one = torch.ones(1, device="cuda")
+    for scale_a, scale_b in ((1.0, 1.0), (2.2, 2.2), (8.0, 8.0)):
+        Aq = np.clip(np.rint(rng.standard_normal((M, K)) * scale_a), -8, 7).astype(np.int8)
+        Bq = np.clip(np.rint(rng.standard_normal((N, K)) * scale_b), -8, 7).astype(np.int8)
+        want_out, want_S, want_tiles = O.gemm_i8_tiled(Aq, Bq, 1.0, 1.0, want_tiles=True)
+        clamped = float(np.mean((want_tiles == 127) | (want_tiles == -128)))
+        _, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), one, one, want_S=True, flags=hdqt.FLAG_NO_MERGE)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), (scale_a, clamped)
+    assert clamped > 0.2                                   # the last case really saturates often
+    for acc_bits in (6, 4, 2):                             # narrower accumulators through the same epilogue
+        want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 1.0, 1.0, acc_bits)
+        _, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), one, one, acc_bits, want_S=True, flags=hdqt.FLAG_NO_MERGE)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), acc_bits
+
+
+def test_bounded_waits_run_out_and_report_timeout(hdqt):
+    """A wait on a barrier nothing arrives at gives up, the block ends normally and the status word holds
+    HDQT_ERR_TIMEOUT; the status word is a sticky maximum; the context stays usable."""
+    status = hdqt.new_status("cuda")
+    gave_up = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    assert hdqt.lib.hdqt_selftest_bounded_wait(status.data_ptr(), gave_up.data_ptr(), stream) == 0
+    torch.cuda.synchronize()
+    assert status.item() == 6 and hdqt.STATUS_NAMES[6] == "TIMEOUT"
+    assert gave_up.item() == 33                            # the spinning thread and the 32 suspending ones
+    with pytest.raises(hdqt.HdqtError) as err:
+        hdqt.check_device_status(status, "selftest")
+    assert err.value.status == 6
+    # sticky maximum: a smaller code (non-finite operand = 5) does not overwrite it, a larger one would
+    z = torch.full((4, 32), float("nan"), device="cuda")
+    hdqt.quantize_hadamard(z, dev_status=status)
+    assert status.item() == 6
+    status.zero_()
+    hdqt.quantize_hadamard(z, dev_status=status)
+    assert status.item() == 5
+    # the device is still fine: a real GEMM afterwards gives the right answer
+    A = np.full((8, 32), 1, np.int8)
+    one = torch.ones(1, device="cuda")
+    _, S, _ = hdqt.gemm_i8_tiled(_dev(A), _dev(A), one, one, want_S=True)
+    assert (S == 32).all().item()

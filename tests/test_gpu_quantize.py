@@ -103,8 +103,13 @@ def test_all_zero_and_nonfinite(hdqt):
     codes, step, _ = hdqt.quantize_hadamard(z, dev_status=status)
     assert not codes.any().item() and step.item() == 0.0 and status.item() == 0
     z[3, 5] = float("inf")
-    hdqt.quantize_hadamard(z, dev_status=status)
-    assert status.item() == 5          # HDQT_ERR_NONFINITE, reported through the device status word
+    for src in (z, z.t().contiguous().t()):
+        for mode in (0, 1):
+            status.zero_()
+            codes, step, _ = hdqt.quantize_hadamard(src, mode=mode, dev_status=status)
+            assert status.item() == 5      # HDQT_ERR_NONFINITE, reported through the device status word
+            # a contaminated operand yields all-zero codes and a zero scale, never saturated garbage
+            assert not codes.any().item() and step.item() == 0.0
     status.zero_()
     z[3, 5] = float("nan")
     hdqt.absmax_hadamard(z.t().contiguous().t(), dev_status=status)
@@ -136,3 +141,16 @@ def test_large_tensor_multiple_waves(hdqt):
             codes, step, _ = hdqt.quantize_hadamard(src, mode=mode, seed=2, tag=4)
             assert step.item() == float(step_w)
             assert np.array_equal(codes.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("bits,clip", [(8, 0.25), (8, 1.0), (7, 0.05), (4, 1.0 / 64)])
+def test_tile_norms_of_wide_and_saturated_codes(hdqt, bits, clip):
+    """Tile norms of 7/8-bit codes reach 32 * 128^2 (far beyond 16 bits); a small clip saturates most codes.
+    Both layouts, several 128-row blocks, a ragged last block and K segments of every width."""
+    for rows, K in ((300, 561), (130, 8192), (257, 96)):
+        x = inputs.activations(rows, K, seed=bits + rows)
+        want_codes, _, _ = O.quantize_hadamard(x, 32, bits, clip, 0)
+        for src in (_dev(x), _dev(x.T).t()):
+            codes, _, norms = hdqt.quantize_hadamard(src, 32, bits, clip, 0, want_norms=True)
+            assert np.array_equal(codes.cpu().numpy(), want_codes)
+            assert np.array_equal(norms.cpu().numpy().astype(np.int64), _expected_norms(want_codes))
