@@ -52,7 +52,7 @@ def needs_rebuild() -> bool:
 
 
 def _compile(out_path: str, defines=(), verbose: bool = False) -> None:
-    cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
+    cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++20", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     cmd += [f"-D{d}" for d in defines]

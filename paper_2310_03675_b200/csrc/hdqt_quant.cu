@@ -34,7 +34,9 @@ __device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x
 // ---- butterflies ------------------------------------------------------------------------
 
 // strides 1, 2, 4 on 8 register values (only those below had_block)
+template <bool kHad32 = false>
 __device__ __forceinline__ void fwht8_regs(float (&x)[8], int had_block) {
+  if (kHad32) had_block = 32;
   if (had_block > 1) {
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
@@ -66,7 +68,9 @@ __device__ __forceinline__ void fwht8_regs(float (&x)[8], int had_block) {
 // strides 8 and 16 across lanes (lane^1, lane^2); the whole warp must call this.
 // The lower lane of a pair needs x + y, the upper one y - x: both are fma(sign, x, y) with sign = +-1
 // (sign*x is exact, so the fused form rounds once, exactly like the add / subtract).
+template <bool kHad32 = false>
 __device__ __forceinline__ void fwht8_lanes(float (&x)[8], int had_block, int lane) {
+  if (kHad32) had_block = 32;
   if (had_block > 8) {
     const float sign = (lane & 1) ? -1.0f : 1.0f;
 #pragma unroll
@@ -86,7 +90,9 @@ __device__ __forceinline__ void fwht8_lanes(float (&x)[8], int had_block, int la
 }
 
 // all stages on 32 register values
+template <bool kHad32 = false>
 __device__ __forceinline__ void fwht32_regs(float (&x)[32], int had_block) {
+  if (kHad32) had_block = 32;
 #pragma unroll
   for (int h = 1; h < 32; h <<= 1) {
     if (h < had_block) {
@@ -144,11 +150,14 @@ __device__ __forceinline__ uint32_t pack4_offset(const int (&t)[8], int base, ui
   return (w + addc) ^ 0x80808080u;
 }
 
-// codes of 8 consecutive elements as two packed words; `g` = (linear index of the first element) / 8
+// codes of 8 consecutive elements as two packed words; `g` = (linear index of the first element) / 8.
+// kMode: 0 = nearest, 1 = stochastic with the fixed-point conversion through the fp32 adder (|v| < 64
+// guaranteed), 2 = stochastic with a float-to-int conversion (any v; a quarter of the arithmetic rate).
+template <int kMode>
 __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams& p, uint64_t g, uint32_t& w0,
                                           uint32_t& w1) {
   int t[8];
-  if (p.mode == HDQT_ROUND_NEAREST) {
+  if (kMode == 0) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float v = __fmul_rn(x[i], p.m);
@@ -158,24 +167,41 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams
     }
   } else {
     const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, 0u, *p.keys);
+    // s = rint(v * 2^16) + u16 + (offset << 16), a Q.16 fixed-point integer; code + offset = floor(s / 2^16), clamped
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float v = __fmul_rn(x[i], p.m);
       const uint32_t word = rnd.w[i >> 1];
       const int u16 = (i & 1) ? (int)(word >> 16) : (int)(word & 0xFFFFu);
-      int s;  // rint(v * 2^16) + u16 + (offset << 16), a Q.16 fixed-point integer
-      if (p.sr_magic) {
+      int s;
+      if (kMode == 1) {
         // for v in [-64, 64): v + 192 lies in [128, 256) where one ulp is 2^-16
         s = __float_as_int(__fadd_rn(v, 192.0f)) + u16 + p.sr_bias;
       } else {
         s = __float2int_rn(__fmul_rn(v, 65536.0f)) + u16 + p.off16;
       }
-      t[i] = __vimin_s32_relu(s >> 16, p.rng);   // floor((v_fx + u16) / 2^16) + offset, clamped
+      t[i] = __vimin_s32_relu(s >> 16, p.rng);
     }
   }
   w0 = pack4_offset(t, 0, p.addc);
   w1 = pack4_offset(t, 4, p.addc);
   if (p.zero_all) { w0 = 0u; w1 = 0u; }
+}
+
+// Runs `body.template operator()<kMode, kHad32>()` for the operand's rounding mode and Hadamard block: the
+// per-chunk code is then free of mode and block-size tests (they cost more than a tenth of its instructions).
+template <typename Body>
+__device__ __forceinline__ void dispatch_mode(const QuantParams& p, int had_block, Body body) {
+  const int mode = (p.mode == HDQT_ROUND_NEAREST) ? 0 : (p.sr_magic ? 1 : 2);
+  if (had_block == 32) {
+    if (mode == 0) body.template operator()<0, true>();
+    else if (mode == 1) body.template operator()<1, true>();
+    else body.template operator()<2, true>();
+  } else {
+    if (mode == 0) body.template operator()<0, false>();
+    else if (mode == 1) body.template operator()<1, false>();
+    else body.template operator()<2, false>();
+  }
 }
 
 __device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bits, float clip, int mode,
@@ -354,7 +380,7 @@ absmax_kc_kernel(const __grid_constant__ QuantBatch b, int32_t* dev_status) {
 }
 
 // quantize, linear mapping (no tile norms)
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__ PhiloxKeys keys,
                    int32_t* dev_status) {
   int local_block;
@@ -371,6 +397,7 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
   const bool dense = (K == op.K_pad) && (ld_row == K);
   const int lane = threadIdx.x & 31;
+  auto body = [&]<int kMode, bool kHad32>() {
   for (int64_t base = (int64_t)local_block * (kThreads * kUnrollQuant); base < total;
        base += (int64_t)op.num_blocks * (kThreads * kUnrollQuant)) {
     float x[kUnrollQuant][8];
@@ -393,21 +420,23 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
 #pragma unroll
     for (int u = 0; u < kUnrollQuant; ++u) {
       const int64_t c = base + u * kThreads + threadIdx.x;
-      fwht8_regs(x[u], had_block);
-      fwht8_lanes(x[u], had_block, lane);
+      fwht8_regs<kHad32>(x[u], had_block);
+      fwht8_lanes<kHad32>(x[u], had_block, lane);
       uint2 out;
-      quantize8(x[u], p, (uint64_t)c, out.x, out.y);  // linear index of the chunk's first element is 8*c
+      quantize8<kMode>(x[u], p, (uint64_t)c, out.x, out.y);  // linear index of the chunk's first element is 8*c
       // codes are dense [rows, K_pad]: chunk c is bytes [8c, 8c+8)
       if (c < total) *reinterpret_cast<uint2*>(codes + (c << 3)) = out;
     }
   }
+  };
+  dispatch_mode(p, had_block, body);
 }
 
 // quantize, blocked mapping, with the tile norms: a work item is 128 rows x one K segment of 2^seg_log2
 // elements (32..256), so that the maximum over the 128 rows of every tile's sum(code^2) is formed inside
 // the thread block and written once.  A row's segment is covered by seg/8 neighbouring lanes; a warp
 // covers 32/(seg/8) rows per pass, the block's 8 warps cover consecutive rows.
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__ PhiloxKeys keys,
                          int32_t* dev_status) {
   __shared__ int s_norm[kThreads / 32][32];
@@ -430,40 +459,78 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
   const int64_t T = K_pad >> 5;
   const int64_t cpr = K_pad >> 3;                // chunks per code row
   const int64_t n_items = ((rows + 127) >> 7) * nseg;
+  auto body = [&]<int kMode, bool kHad32>() {
   for (int64_t item = local_block; item < n_items; item += op.num_blocks) {
     const int64_t rb = item / nseg, kseg = item - rb * nseg;
     const int64_t k0 = (kseg << op.seg_log2) + (kc << 3);
     const bool k_ok = k0 < K_pad;
     int nmax = 0;
-    for (int pass = 0; pass < passes; pass += kUnrollQuant) {
-      float x[kUnrollQuant][8];
-      int64_t r[kUnrollQuant];
+    const int64_t row0 = (rb << 7) + warp * rpw + row_sub;    // this thread's row in pass 0; a pass adds 8 * rpw rows
+    const bool whole = vec && ((rb << 7) + 128 <= rows) && (((kseg + 1) << op.seg_log2) <= K);
+    if (whole) {
+      // whole 128-row block, whole segment inside K, vector loads: nothing to test per chunk, running pointers
+      const float* __restrict__ sp = src + row0 * ld_row + k0;
+      int8_t* __restrict__ cp = codes + row0 * K_pad + k0;
+      uint64_t g = (uint64_t)row0 * (uint64_t)cpr + (uint64_t)(k0 >> 3);
+      const int64_t s_step = 8 * (int64_t)rpw * ld_row, c_step = 8 * (int64_t)rpw * K_pad;
+      const uint64_t g_step = 8ull * (uint64_t)rpw * (uint64_t)cpr;
+      for (int pass = 0; pass < passes; pass += kUnrollQuant) {
+        float x[kUnrollQuant][8];
 #pragma unroll
-      for (int u = 0; u < kUnrollQuant; ++u) {
-        r[u] = (rb << 7) + (int64_t)((pass + u) * 8 + warp) * rpw + row_sub;
-        if (k_ok && pass + u < passes && r[u] < rows) {
-          load8_kc(src + r[u] * ld_row, k0, K, vec, x[u]);
-        } else {
-          r[u] = -1;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) x[u][i] = 0.0f;
+        for (int u = 0; u < kUnrollQuant; ++u) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(sp + u * s_step));
+          const float4 c = __ldg(reinterpret_cast<const float4*>(sp + u * s_step + 4));
+          x[u][0] = a.x; x[u][1] = a.y; x[u][2] = a.z; x[u][3] = a.w;
+          x[u][4] = c.x; x[u][5] = c.y; x[u][6] = c.z; x[u][7] = c.w;
         }
-      }
 #pragma unroll
-      for (int u = 0; u < kUnrollQuant; ++u) {
-        fwht8_regs(x[u], had_block);
-        fwht8_lanes(x[u], had_block, lane);
-        const bool valid = r[u] >= 0;
-        const uint64_t g = valid ? (uint64_t)r[u] * (uint64_t)cpr + (uint64_t)(k0 >> 3) : 0u;
-        uint2 out;
-        quantize8(x[u], p, g, out.x, out.y);
-        int ss = __dp4a((int)out.x, (int)out.x, 0);
-        ss = __dp4a((int)out.y, (int)out.y, ss);
-        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
-        ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
-        if (valid) {
+        for (int u = 0; u < kUnrollQuant; ++u) {
+          fwht8_regs<kHad32>(x[u], had_block);
+          fwht8_lanes<kHad32>(x[u], had_block, lane);
+          uint2 out;
+          quantize8<kMode>(x[u], p, g + u * g_step, out.x, out.y);
+          int ss = __dp4a((int)out.x, (int)out.x, 0);
+          ss = __dp4a((int)out.y, (int)out.y, ss);
+          ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+          ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
           nmax = max(nmax, ss);
-          *reinterpret_cast<uint2*>(codes + r[u] * K_pad + k0) = out;
+          *reinterpret_cast<uint2*>(cp + u * c_step) = out;
+        }
+        sp += kUnrollQuant * s_step;
+        cp += kUnrollQuant * c_step;
+        g += kUnrollQuant * g_step;
+      }
+    } else {
+      for (int pass = 0; pass < passes; pass += kUnrollQuant) {
+        float x[kUnrollQuant][8];
+        int64_t r[kUnrollQuant];
+#pragma unroll
+        for (int u = 0; u < kUnrollQuant; ++u) {
+          r[u] = row0 + (int64_t)(pass + u) * 8 * rpw;
+          if (k_ok && r[u] < rows) {
+            load8_kc(src + r[u] * ld_row, k0, K, vec, x[u]);
+          } else {
+            r[u] = -1;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[u][i] = 0.0f;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnrollQuant; ++u) {
+          fwht8_regs<kHad32>(x[u], had_block);
+          fwht8_lanes<kHad32>(x[u], had_block, lane);
+          const bool valid = r[u] >= 0;
+          const uint64_t g = valid ? (uint64_t)r[u] * (uint64_t)cpr + (uint64_t)(k0 >> 3) : 0u;
+          uint2 out;
+          quantize8<kMode>(x[u], p, g, out.x, out.y);
+          int ss = __dp4a((int)out.x, (int)out.x, 0);
+          ss = __dp4a((int)out.y, (int)out.y, ss);
+          ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+          ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+          if (valid) {
+            nmax = max(nmax, ss);
+            *reinterpret_cast<uint2*>(codes + r[u] * K_pad + k0) = out;
+          }
         }
       }
     }
@@ -480,6 +547,8 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
     }
     __syncthreads();
   }
+  };
+  dispatch_mode(p, had_block, body);
 }
 
 // ---- K-strided kernels ------------------------------------------------------------------------
@@ -543,6 +612,7 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   const uint32_t row_groups = (uint32_t)((rows + kThreads - 1) / kThreads);
   const uint32_t items = row_groups * (uint32_t)T;   // the host guarantees that this fits 31 bits
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  auto body = [&]<int kMode, bool kHad32>() {
   for (uint32_t item = (uint32_t)local_block; item < items; item += (uint32_t)op.num_blocks) {
     const uint32_t kbu = item / row_groups;     // uniform over the block
     const int64_t kb = kbu;
@@ -552,7 +622,7 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
     if (r < rows) {
       float x[32];
       load32_ks(src, r, kb, K, ld_k, x);
-      fwht32_regs(x, had_block);
+      fwht32_regs<kHad32>(x, had_block);
       uint32_t w[8];
       const uint64_t g0 = (uint64_t)(r * K_pad + (kb << 5)) >> 3;
 #pragma unroll
@@ -560,7 +630,7 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
         float x8[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) x8[i] = x[8 * j + i];
-        quantize8(x8, p, g0 + j, w[2 * j], w[2 * j + 1]);
+        quantize8<kMode>(x8, p, g0 + j, w[2 * j], w[2 * j + 1]);
         ss = __dp4a((int)w[2 * j], (int)w[2 * j], ss);
         ss = __dp4a((int)w[2 * j + 1], (int)w[2 * j + 1], ss);
       }
@@ -584,6 +654,8 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
       }
     }
   }
+  };
+  dispatch_mode(p, had_block, body);
 }
 
 constexpr int kMaxDevices = 64;
