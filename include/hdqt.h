@@ -69,7 +69,8 @@ typedef enum {
 } hdqt_round_t;
 
 /* flags for the GEMM entry points */
-#define HDQT_FLAG_NO_MERGE 1u /* never merge provably clamp-free tiles (see hdqt_gemm_i8_tiled) */
+#define HDQT_FLAG_NO_MERGE 1u   /* never merge provably clamp-free tiles (see hdqt_gemm_i8_tiled) */
+#define HDQT_FLAG_NO_SPLIT_K 2u /* never cut a long contraction with few output blocks into several work items */
 
 /*
  * Parameters of one HDQT GEMM Out[M,N] = A[M,K] B[K,N] (Section 3).

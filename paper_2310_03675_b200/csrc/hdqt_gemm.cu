@@ -80,6 +80,19 @@ __global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(int32_t* dev_
   if (threadIdx.x == 0 && abort_flag) report_status(dev_status, HDQT_ERR_TIMEOUT);
 }
 
+// ---- split-K: integer sums parked in the output buffer -> fp32 result (and optional integer output) ----
+__global__ void split_k_finalize_kernel(const GemmParams p) {
+  const float scale = dequant_scale(p);
+  const int64_t total = p.M * p.N;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t m = i / p.N, n = i - m * p.N;
+    float* o = p.out + m * p.ld_out + n;
+    const int S = __float_as_int(*o);
+    *o = __fmul_rn((float)S, scale);
+    if (p.S_out != nullptr) p.S_out[i] = S;
+  }
+}
+
 // ---- host side --------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -234,8 +247,35 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
   const int64_t num_blocks = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   if (num_blocks > INT32_MAX) return HDQT_ERR_UNSUPPORTED;
   const int sms = sm_count();
-  dim3 grid((unsigned)(num_blocks < sms ? num_blocks : sms));   // persistent: one CTA per SM
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+  // Split-K: a long contraction with few output blocks (the weight gradient of a convolution: K = batch x
+  // positions) would leave most SMs idle.  Only where every tile takes the clamp path anyway (no merging), in
+  // whole shared-memory stages and whole accumulator tiles; with the 16-bit-lane epilogue a work item stays
+  // within one widening period.  Integer addition is exact and order-free, so the result is unchanged.
+  p.split_k = 1;
+  p.split_kblocks = 0;
+  if (p.merge == 0 && !tiles_out && num_blocks * 2 <= sms && (flags & HDQT_FLAG_NO_SPLIT_K) == 0) {
+    const int64_t unit = (tpa % 4 == 0) ? tpa : ((tpa % 2 == 0) ? 2 * tpa : 4 * tpa);   // lcm(4, tpa) tiles
+    const int64_t units = tiles32 / unit;                                              // whole units in K
+    int64_t want = sms / num_blocks;
+    // at least 8 stages per item (the fixed cost of an item is a few tiles' worth), at most `want` items
+    int64_t per_item = (units + want - 1) / want;
+    const int64_t min_units = (32 + unit - 1) / unit;
+    if (per_item < min_units) per_item = min_units;
+    if (packed && per_item * unit > (int64_t)p.flush_every * tpa) per_item = (int64_t)p.flush_every * tpa / unit;
+    const int64_t items = per_item > 0 ? (tiles32 + per_item * unit - 1) / (per_item * unit) : 1;
+    if (per_item > 0 && items > 1 && items <= 65535) {
+      p.split_k = (int32_t)items;
+      p.split_kblocks = (int32_t)(per_item * unit / 4);
+    }
+  }
+  const int64_t num_items = num_blocks * p.split_k;
+  dim3 grid((unsigned)(num_items < sms ? num_items : sms));   // persistent: one CTA per SM
+  if (p.split_k > 1) {
+    if (cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0, (size_t)N * sizeof(float), (size_t)M, s) != cudaSuccess)
+      return HDQT_ERR_CUDA;
+  }
 
   // Large problems (at least 8 output blocks per SM; below that the extra launches cost more than they gain)
   // with clamp-free tiles: the cta_group::2 kernel takes the blocks whose K tiles are all, or all but a few,
@@ -281,9 +321,17 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
     return acc_shift ? launch_variant<false, true, true>(ma, mb, p, grid, s)
                      : launch_variant<false, false, true>(ma, mb, p, grid, s);
   }
-  if (packed) return launch_variant<true, false, false>(ma, mb, p, grid, s);
-  return acc_shift ? launch_variant<false, true, false>(ma, mb, p, grid, s)
-                   : launch_variant<false, false, false>(ma, mb, p, grid, s);
+  hdqt_status_t st;
+  if (packed) st = launch_variant<true, false, false>(ma, mb, p, grid, s);
+  else st = acc_shift ? launch_variant<false, true, false>(ma, mb, p, grid, s)
+                      : launch_variant<false, false, false>(ma, mb, p, grid, s);
+  if (st == HDQT_OK && p.split_k > 1) {
+    const int64_t total = M * N;
+    const int64_t blocks = (total + 255) / 256;
+    split_k_finalize_kernel<<<(unsigned)(blocks < 4 * sms ? blocks : 4 * sms), 256, 0, s>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return HDQT_ERR_CUDA;
+  }
+  return st;
 }
 
 extern "C" hdqt_status_t hdqt_calibrate_acc_shift(const int8_t* Aq, const int8_t* Bq, int64_t M, int64_t N,

@@ -77,6 +77,8 @@ struct GemmParams {
   int32_t had_block;
   int32_t flush_every;    // packed mode: accumulator tiles summed in 16-bit lanes before widening
   int32_t offset_mma;     // packed mode: every clamp-path accumulator tile starts from the constant 2^(b_a-1)
+  int32_t split_k;        // > 1: the contraction of every output block is cut into this many work items
+  int32_t split_kblocks;  // shared-memory stages (4 tiles of 32) per work item
   // merging of provably clamp-free accumulator tiles
   int32_t merge;          // 0 = off, 1 = certificates from the tile norms, 2 = every tile is clamp-free
   int32_t merge_max_uncert_256;  // a CTA merges only if uncertified tiles <= this/256 of all tiles
@@ -406,10 +408,11 @@ struct EpiCtx {               // constants of one epilogue warp
 };
 
 struct BlockJob {             // one output block as seen by the epilogue
-  int m0, n0;
-  int n_clamp_tiles;          // accumulator tiles that arrive one by one for the clamp path
-  int n_merged;               // accumulator tiles merged in accumulator 0
-  int merging;                // clamp tiles use accumulator 1 only (else they alternate 0 / 1)
+  int m0 = 0, n0 = 0;
+  int n_clamp_tiles = 0;      // accumulator tiles that arrive one by one for the clamp path
+  int n_merged = 0;           // accumulator tiles merged in accumulator 0
+  int merging = 0;            // clamp tiles use accumulator 1 only (else they alternate 0 / 1)
+  int atomic = 0;             // split-K: add the integer sums into the output buffer instead of storing the result
 };
 
 __device__ __forceinline__ float dequant_scale(const GemmParams& p) {
@@ -426,6 +429,16 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
                                             int (&val)[16], bool parked, float scale, bool raw = false) {
   const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
   const int64_t gn = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16;
+  if (job.atomic) {
+    // split-K: integer partial sums of this K range (the buffer was cleared before the launch)
+    if (gm < p.M) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        if (gn + i < p.N && val[i] != 0) atomicAdd(reinterpret_cast<int*>(p.out + gm * p.ld_out + gn + i), val[i]);
+      }
+    }
+    return;
+  }
   const bool staged = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
                       (gn + 16 <= p.N);    // warp-uniform
   if (staged) {

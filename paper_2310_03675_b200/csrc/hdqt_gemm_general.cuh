@@ -84,6 +84,23 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   const int num_kblocks = (p.tiles32 + 3) >> 2;
   const int num_acc = p.num_acc;
   if (num_tiles == 0) return;   // an empty work list (uniform over the grid): nothing to set up or tear down
+  // Split-K (host-selected for long contractions with few output blocks, clamp path only): a work item is then
+  // (output block, K range of split_kblocks stages); the integer sums of the ranges are added up in the output
+  // buffer with atomics (exact and order-free) and a small kernel applies the scale afterwards.
+  const int split_k = p.split_k > 1 ? p.split_k : 1;
+  const int num_items = num_tiles * split_k;
+  struct ItemRange { int blk, kb_lo, kb_hi, t_end, n_acc; };
+  auto item_range = [&](int item) {
+    ItemRange r{item, 0, num_kblocks, p.tiles32, num_acc};
+    if (split_k > 1) {
+      r.blk = item / split_k;
+      r.kb_lo = (item - r.blk * split_k) * p.split_kblocks;
+      r.kb_hi = min(num_kblocks, r.kb_lo + p.split_kblocks);
+      r.t_end = min(p.tiles32, r.kb_hi * 4);
+      r.n_acc = (r.t_end - r.kb_lo * 4 + p.tiles_per_acc - 1) / p.tiles_per_acc;
+    }
+    return r;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -137,10 +154,11 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     if (lane == 0) {
       uint32_t it = 0;   // k-blocks issued so far, over all output blocks
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int tile = blockIdx.x; tile < num_items && ok; tile += gridDim.x) {
+        const ItemRange ir = item_range(tile);
         int tile_m, tile_n;
-        block_coords(p, tile, tiles_m, tiles_n, tile_m, tile_n);
-        for (int kb = 0; kb < num_kblocks; ++kb, ++it) {
+        block_coords(p, ir.blk, tiles_m, tiles_n, tile_m, tile_n);
+        for (int kb = ir.kb_lo; kb < ir.kb_hi; ++kb, ++it) {
           const uint32_t s = it % STAGES;
           const uint32_t par = ((it / STAGES) & 1u) ^ 1u;
           if (!mbar_wait_suspend(bar_empty + 8 * s, par, abort_flag)) { ok = false; break; }
@@ -225,10 +243,13 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       uint32_t fills[2] = {0u, 0u};   // how many times each TMEM accumulator has been handed to the epilogue
       uint64_t desc_a = desc_a0, desc_b = desc_b0;
       bool ok = true;
-      const int tiles32 = p.tiles32, tpa = p.tiles_per_acc;
+      const int tpa = p.tiles_per_acc;
       bool ready = false;
       int ti = 0;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ti) {
+      for (int tile = blockIdx.x; tile < num_items && ok; tile += gridDim.x, ++ti) {
+        const ItemRange ir = item_range(tile);
+        const int tiles32 = ir.t_end;      // end of this item's K range, in 32-wide tiles
+        const int num_acc = ir.n_acc;      // (shadows the block-wide count: accumulator tiles of this item)
         const int slot = ti & 1;
         int n_uncert = (p.merge == 2) ? 0 : num_acc;
         if (p.merge == 1) {
@@ -246,7 +267,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         uint32_t merged_started = 0;
         uint32_t d_tmem = tmem_base;
         int cur_buf = 0;
-        for (int kb = 0; kb < num_kblocks; ++kb) {
+        for (int kb = ir.kb_lo; kb < ir.kb_hi; ++kb) {
           if (!ready && !mbar_wait(bar_full + 8 * s, full_par, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t s_next = (s + 1 == STAGES) ? 0u : s + 1;
@@ -371,19 +392,21 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     e.box = reinterpret_cast<float*>(smem_al + OUT_STAGE_OFF + (warp - NUM_CTRL_WARPS) * OUT_STAGE_WARP);
     uint32_t drains[2] = {0u, 0u};      // how many times this warp has drained each accumulator
     int ti = 0;
-    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++ti) {
+    for (int tile = blockIdx.x; tile < num_items; tile += gridDim.x, ++ti) {
+      const ItemRange ir = item_range(tile);
       const int slot = ti & 1;
-      int n_uncert = (p.merge == 2) ? 0 : num_acc;
+      int n_uncert = (p.merge == 2) ? 0 : ir.n_acc;
       if (p.merge == 1) {
         if (!mbar_wait_yield<128>(bar_ifull + 8 * slot, ((uint32_t)ti >> 1) & 1u, abort_flag)) break;
         n_uncert = *reinterpret_cast<volatile int32_t*>(&tile_info[slot].n_uncert);
       }
       BlockJob job;
       job.merging = block_merges(n_uncert) ? 1 : 0;
-      job.n_clamp_tiles = job.merging ? n_uncert : num_acc;
-      job.n_merged = job.merging ? num_acc - n_uncert : 0;
+      job.n_clamp_tiles = job.merging ? n_uncert : ir.n_acc;
+      job.n_merged = job.merging ? ir.n_acc - n_uncert : 0;
+      job.atomic = split_k > 1 ? 1 : 0;
       int tile_m, tile_n;
-      block_coords(p, tile, tiles_m, tiles_n, tile_m, tile_n);
+      block_coords(p, ir.blk, tiles_m, tiles_n, tile_m, tile_n);
       job.m0 = tile_m * BM;
       job.n0 = tile_n * BN;
       bool ok;

@@ -17,6 +17,7 @@ from . import build as _build
 ROUND_NEAREST = 0
 ROUND_STOCHASTIC = 1
 FLAG_NO_MERGE = 1
+FLAG_NO_SPLIT_K = 2
 
 STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "WORKSPACE", "NONFINITE", "TIMEOUT", "CUDA",
                 "STATIC_SCRATCH"]

@@ -119,3 +119,264 @@ def train_step(model: Mlp, opt: torch.optim.Optimizer, x, labels, step: int):
     loss.backward()
     opt.step()
     return loss
+
+
+# ---- convolution as an im2col GEMM -------------------------------------------------------------------
+# The transform and the quantizer act along the contraction dimension of the matmul a convolution lowers to
+# (paper Section 3: Z = X W for every layer): rows = output positions (batch x Ho x Wo), contraction =
+# Cin x kh x kw, columns = output channels.
+
+# Layout: activations are handled as NHWC (the channels-last storage of a [B, C, H, W] tensor), and the
+# contraction index runs over (kh, kw, cin) with cin fastest, so that every 32-wide Hadamard block / accumulator
+# tile of a layer with cin % 32 == 0 is 32 consecutive channels of one input pixel.
+
+def _nhwc(x):
+    """[B, C, H, W] (any strides) -> contiguous [B, H, W, C] (no copy for channels-last tensors)."""
+    return x.permute(0, 2, 3, 1).contiguous()
+
+
+def _im2col(x, kernel, stride, padding):
+    """x [B, Cin, H, W] -> (X_col [B*Ho*Wo, kh*kw*Cin] contiguous, Ho, Wo): one strided copy per kernel tap."""
+    B, C, H, W = x.shape
+    Ho = (H + 2 * padding - kernel) // stride + 1
+    Wo = (W + 2 * padding - kernel) // stride + 1
+    xn = _nhwc(x)
+    if kernel == 1 and padding == 0:
+        return xn[:, ::stride, ::stride, :].reshape(B * Ho * Wo, C), Ho, Wo
+    if padding:
+        xn = torch.nn.functional.pad(xn, (0, 0, padding, padding, padding, padding))
+    cols = torch.empty((B, Ho, Wo, kernel * kernel, C), dtype=x.dtype, device=x.device)
+    for kh in range(kernel):
+        for kw in range(kernel):
+            cols[:, :, :, kh * kernel + kw, :] = xn[:, kh:kh + (Ho - 1) * stride + 1:stride,
+                                                    kw:kw + (Wo - 1) * stride + 1:stride, :]
+    return cols.view(B * Ho * Wo, kernel * kernel * C), Ho, Wo
+
+
+def _col2im(dcols, xshape, kernel, stride, padding, Ho, Wo):
+    """Adjoint of _im2col: dX_col [B*Ho*Wo, kh*kw*Cin] -> dX as a channels-last [B, Cin, H, W] tensor."""
+    B, C, H, W = xshape
+    d = dcols.view(B, Ho, Wo, kernel * kernel, C)
+    if kernel == 1 and padding == 0:
+        if stride == 1:
+            return d.view(B, H, W, C).permute(0, 3, 1, 2)
+        dx = torch.zeros((B, H, W, C), dtype=dcols.dtype, device=dcols.device)
+        dx[:, ::stride, ::stride, :] = d[:, :, :, 0, :]
+        return dx.permute(0, 3, 1, 2)
+    dx = torch.zeros((B, H + 2 * padding, W + 2 * padding, C), dtype=dcols.dtype, device=dcols.device)
+    for kh in range(kernel):
+        for kw in range(kernel):
+            dx[:, kh:kh + (Ho - 1) * stride + 1:stride, kw:kw + (Wo - 1) * stride + 1:stride, :] += d[:, :, :, kh * kernel + kw, :]
+    return dx[:, padding:padding + H, padding:padding + W, :].permute(0, 3, 1, 2)
+
+
+def _weight_matrix(w):
+    """[Cout, Cin, kh, kw] -> [Cout, kh*kw*Cin] in the contraction order of _im2col (the "[C, D]" weight layout)."""
+    return w.permute(0, 2, 3, 1).reshape(w.shape[0], -1)
+
+
+class HdqtConv2dFunction(torch.autograd.Function):
+    """y = conv2d(x, w) (no bias) with the forward, dX and dW products as HDQT GEMMs on the im2col matrix."""
+
+    @staticmethod
+    def forward(ctx, x, w, stride: int, padding: int, layer_id: int, seed: int, over: dict):
+        B, Cin, H, W = x.shape
+        Cout, _, kh, kw = w.shape
+        xc, Ho, Wo = _im2col(x, kh, stride, padding)
+        wm = _weight_matrix(w).contiguous()
+        d = _desc("fwd", layer_id, seed, **over)
+        y2d, _ = hdqt.gemm_fwd(xc, wm, desc=d, w_is_cd=True,
+                               workspace=_workspace(d, xc.shape[0], Cout, xc.shape[1], x.device))
+        ctx.save_for_backward(xc, wm)
+        ctx.meta = (layer_id, seed, over, (B, Cin, H, W), (Cout, Cin, kh, kw), stride, padding, Ho, Wo)
+        # [B*Ho*Wo, Cout] is the channels-last storage of [B, Cout, Ho, Wo]: no copy
+        return y2d.view(B, Ho, Wo, Cout).permute(0, 3, 1, 2)
+
+    @staticmethod
+    def backward(ctx, g):
+        xc, wm = ctx.saved_tensors
+        layer_id, seed, over, xshape, wshape, stride, padding, Ho, Wo = ctx.meta
+        B = xshape[0]
+        Cout, Cin, kh, kw = wshape
+        g2d = _nhwc(g).view(B * Ho * Wo, Cout)
+        dx = dw = None
+        if ctx.needs_input_grad[0]:
+            d = _desc("dgrad", layer_id, seed, **over)
+            dxc, _ = hdqt.gemm_dgrad(g2d, wm, desc=d, w_is_cd=True,
+                                     workspace=_workspace(d, g2d.shape[0], wm.shape[1], Cout, g.device))
+            dx = _col2im(dxc, xshape, kh, stride, padding, Ho, Wo)
+        if ctx.needs_input_grad[1]:
+            d = _desc("wgrad", layer_id, seed, **over)
+            dwm, _ = hdqt.gemm_wgrad(xc, g2d, desc=d, w_is_cd=True,
+                                     workspace=_workspace(d, Cout, wm.shape[1], xc.shape[0], g.device))
+            dw = dwm.view(Cout, kh, kw, Cin).permute(0, 3, 1, 2)
+        return dx, dw, None, None, None, None, None
+
+
+class HdqtConv2d(torch.nn.Module):
+    """3x3 / 1x1 convolution without bias; quantized=False runs torch's fp32 convolution on the same weights."""
+
+    def __init__(self, cin: int, cout: int, kernel: int, stride: int = 1, padding: int = 0, layer_id: int = 0,
+                 quantized: bool = True, **over):
+        super().__init__()
+        self.weight = torch.nn.Parameter(torch.empty(cout, cin, kernel, kernel))
+        torch.nn.init.kaiming_normal_(self.weight, mode="fan_out", nonlinearity="relu")
+        self.stride, self.padding, self.layer_id, self.quantized, self.over = stride, padding, layer_id, quantized, over
+        self.step = 0
+
+    def forward(self, x):
+        if not self.quantized:
+            return torch.nn.functional.conv2d(x, self.weight, None, self.stride, self.padding)
+        return HdqtConv2dFunction.apply(x, self.weight, self.stride, self.padding, self.layer_id, self.step, self.over)
+
+
+class _BasicBlock(torch.nn.Module):
+    def __init__(self, cin, cout, stride, ids, quantized, over):
+        super().__init__()
+        self.conv1 = HdqtConv2d(cin, cout, 3, stride, 1, next(ids), quantized, **over)
+        self.bn1 = torch.nn.BatchNorm2d(cout)
+        self.conv2 = HdqtConv2d(cout, cout, 3, 1, 1, next(ids), quantized, **over)
+        self.bn2 = torch.nn.BatchNorm2d(cout)
+        self.shortcut = None
+        if stride != 1 or cin != cout:
+            self.shortcut = HdqtConv2d(cin, cout, 1, stride, 0, next(ids), quantized, **over)
+            self.bn_sc = torch.nn.BatchNorm2d(cout)
+
+    def forward(self, x):
+        y = torch.relu(self.bn1(self.conv1(x)))
+        y = self.bn2(self.conv2(y))
+        sc = x if self.shortcut is None else self.bn_sc(self.shortcut(x))
+        return torch.relu(y + sc)
+
+
+class ResNet18Width(torch.nn.Module):
+    """ResNet-18-width network for 32x32x3 inputs (3x3 stem, four stages of two basic blocks with 64/128/256/512
+    channels, global average pool, linear head).  Every convolution and the head go through the HDQT GEMMs;
+    batch norm, ReLU, pooling, loss and the optimiser stay in fp32 torch ops.  `num_outputs` is the size of the
+    head; `forward(x, n_seen)` uses only the first n_seen output neurons (a head that grows with the classes seen)."""
+
+    def __init__(self, num_outputs: int = 100, quantized: bool = True, widths=(64, 128, 256, 512), **over):
+        super().__init__()
+        ids = iter(range(1000))
+        self.quantized = quantized
+        self.stem = HdqtConv2d(3, widths[0], 3, 1, 1, next(ids), quantized, **over)
+        self.bn = torch.nn.BatchNorm2d(widths[0])
+        blocks, cin = [], widths[0]
+        for i, w in enumerate(widths):
+            for j in range(2):
+                blocks.append(_BasicBlock(cin, w, 2 if (i > 0 and j == 0) else 1, ids, quantized, over))
+                cin = w
+        self.blocks = torch.nn.ModuleList(blocks)
+        self.head = HdqtLinear(cin, num_outputs, layer_id=next(ids), **over)
+
+    def set_step(self, step: int):
+        for m in self.modules():
+            if isinstance(m, (HdqtConv2d, HdqtLinear)):
+                m.step = step
+
+    def forward(self, x, n_seen: Optional[int] = None):
+        y = torch.relu(self.bn(self.stem(x)))
+        for b in self.blocks:
+            y = b(y)
+        y = y.mean(dim=(2, 3))
+        head = self.head
+        n = head.weight.shape[1] if n_seen is None else n_seen
+        w = head.weight if n == head.weight.shape[1] else head.weight[:, :n].contiguous()
+        if self.quantized:
+            logits = HdqtLinearFunction.apply(y.contiguous(), w, head.layer_id, head.step, head.over)
+        else:
+            logits = y @ w
+        return logits + head.bias[:n]
+
+
+def class_patterns(classes: int, seed: int, device, size: int = 32, waves: int = 4):
+    """One low-frequency pattern per class: a sum of a few 2-D cosines with class-specific frequencies, phases
+    and colour weights, scaled to [0, 1].  Returns [classes, 3, size, size]."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    fx = torch.randint(0, 4, (classes, waves), generator=g, device=device).float()
+    fy = torch.randint(0, 4, (classes, waves), generator=g, device=device).float()
+    ph = torch.rand(classes, waves, generator=g, device=device) * 6.2831853
+    amp = torch.randn(classes, 3, waves, generator=g, device=device)
+    t = torch.arange(size, device=device).float() / size
+    arg = 6.2831853 * (fx[:, :, None, None] * t[None, None, :, None] + fy[:, :, None, None] * t[None, None, None, :]) \
+        + ph[:, :, None, None]                                                  # [classes, waves, size, size]
+    pat = torch.einsum("ckw,cwxy->ckxy", amp, torch.cos(arg))
+    lo = pat.amin(dim=(1, 2, 3), keepdim=True)
+    hi = pat.amax(dim=(1, 2, 3), keepdim=True)
+    return (pat - lo) / (hi - lo + 1e-6)
+
+
+def synthetic_images(labels: torch.Tensor, patterns: torch.Tensor, seed: int, blend: float = 0.5):
+    """Stand-in for 32x32x3 natural images: pixels ~ U[0,1] blended with the label's low-frequency pattern."""
+    g = torch.Generator(device=labels.device)
+    g.manual_seed(seed)
+    noise = torch.rand((labels.numel(),) + tuple(patterns.shape[1:]), generator=g, device=labels.device)
+    return (1.0 - blend) * noise + blend * patterns[labels]
+
+
+def cnn_train_step(model: ResNet18Width, opt, x, labels, step: int, n_seen: Optional[int] = None):
+    model.set_step(step)
+    opt.zero_grad(set_to_none=True)
+    loss = torch.nn.functional.cross_entropy(model(x, n_seen), labels)
+    loss.backward()
+    opt.step()
+    return loss
+
+
+def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_task: int = 20,
+                          steps_per_task: int = 1000, batch: int = 128, memory: int = 2000, seed: int = 0,
+                          lr: float = 0.05, test_per_class: int = 20, log=None, **over):
+    """Plain-replay class-incremental training of the ResNet-18-width model on synthetic classes (paper
+    Section 4: tasks arrive one after the other, a bounded memory of exemplars is replayed, the head grows with
+    the classes seen; appendix: SGD lr 0.05, momentum 0.9, weight decay 2e-4, memory 2000).  Each batch mixes
+    new-task samples and replayed exemplars 1:1.  Returns a dict with the final accuracy over all classes seen,
+    the accuracy after each task and the number of steps taken."""
+    n_classes = tasks * classes_per_task
+    patterns = class_patterns(n_classes, seed, device)
+    torch.manual_seed(seed)
+    model = ResNet18Width(n_classes, quantized=quantized, **over).to(device)
+    opt = torch.optim.SGD(model.parameters(), lr=lr, momentum=0.9, weight_decay=2e-4)
+    g = torch.Generator(device=device)
+    g.manual_seed(seed + 1)
+    mem_x = mem_y = None
+    step = 0
+    acc_after = []
+    test_y = torch.arange(n_classes, device=device).repeat_interleave(test_per_class)
+    test_x = synthetic_images(test_y, patterns, seed=seed + 777)
+    for task in range(tasks):
+        lo, hi = task * classes_per_task, (task + 1) * classes_per_task
+        n_new = batch if mem_x is None else batch // 2
+        model.train()
+        for _ in range(steps_per_task):
+            y = torch.randint(lo, hi, (n_new,), generator=g, device=device)
+            x = synthetic_images(y, patterns, seed=seed + 1000 + step)
+            if mem_x is not None:
+                idx = torch.randint(0, mem_x.shape[0], (batch - n_new,), generator=g, device=device)
+                x = torch.cat([x, mem_x[idx]])
+                y = torch.cat([y, mem_y[idx]])
+            loss = cnn_train_step(model, opt, x, y, step, n_seen=hi)
+            step += 1
+        # exemplar memory: equal quota per class seen so far, random selection
+        quota = memory // hi
+        keep_x, keep_y = [], []
+        if mem_x is not None:
+            for c in range(lo):
+                sel = (mem_y == c).nonzero().flatten()[:quota]
+                keep_x.append(mem_x[sel]); keep_y.append(mem_y[sel])
+        new_y = torch.arange(lo, hi, device=device).repeat_interleave(quota)
+        keep_x.append(synthetic_images(new_y, patterns, seed=seed + 5000 + task)); keep_y.append(new_y)
+        mem_x, mem_y = torch.cat(keep_x), torch.cat(keep_y)
+        # accuracy over every class seen so far
+        model.eval()
+        with torch.no_grad():
+            m = test_y < hi
+            pred = []
+            for i in range(0, int(m.sum()), 500):
+                model.set_step(10 ** 6 + i)
+                pred.append(model(test_x[m][i:i + 500], hi).argmax(1))
+            acc = float((torch.cat(pred) == test_y[m]).float().mean())
+        acc_after.append(acc)
+        if log:
+            log(f"task {task}: loss {float(loss):.3f} accuracy over {hi} classes {acc:.3f}")
+    return {"final_accuracy": acc_after[-1], "accuracy_after_task": acc_after, "steps": step}

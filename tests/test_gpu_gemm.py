@@ -300,9 +300,36 @@ def test_long_contraction_widens_packed_sums(hdqt):
     # odd leading dimension: exercises the scalar store path of the widening too
     big = torch.zeros((M, N + 3), device="cuda")
     for view in (None, big[:, 1:N + 1]):
+        # split-K off: one work item walks all 700 tiles and widens its 16-bit lane sums twice
+        out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), half, eighth, want_S=True, out=view,
+                                       flags=hdqt.FLAG_NO_SPLIT_K)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
+        assert np.array_equal(out.cpu().numpy(), want_out)
+        # split-K on (the default for so few output blocks): same integers, same fp32 values
         out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), half, eighth, want_S=True, out=view)
         assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S)
         assert np.array_equal(out.cpu().numpy(), want_out)
+    assert (big[:, 0] == 0).all().item() and (big[:, N + 1:] == 0).all().item()
+
+
+@pytest.mark.parametrize("acc_bits,acc_tile,acc_shift,K", [(8, 32, 0, 32 * 1001), (8, 96, 0, 32 * 999), (12, 32, 0, 32 * 515),
+                                                           (8, 64, 2, 32 * 640), (6, 32, 0, 32 * 77), (16, 128, 0, 32 * 400)])
+def test_split_k_matches_the_oracle(hdqt, acc_bits, acc_tile, acc_shift, K):
+    """Long contraction, one or two output blocks: the contraction is cut into work items whose integer sums are
+    added up atomically (exact, order-free).  Ragged last item, accumulator tiles of 1, 2, 3 and 4 K tiles, the
+    16-bit-lane and the 32-bit epilogue, with and without a rounding shift, ragged M and N."""
+    rng = np.random.default_rng(K + acc_bits)
+    M, N = 70, 300
+    Aq, Bq = _codes(rng, M, K), _codes(rng, N, K)
+    want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 0.5, 0.25, acc_bits, acc_tile, acc_shift, 32)
+    half, quarter = torch.tensor([0.5], device="cuda"), torch.tensor([0.25], device="cuda")
+    status = hdqt.new_status("cuda")
+    for flags in (0, hdqt.FLAG_NO_SPLIT_K):
+        out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), half, quarter, acc_bits, acc_tile, acc_shift, 32,
+                                       want_S=True, flags=flags, dev_status=status)
+        hdqt.check_device_status(status)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), flags
+        assert np.array_equal(out.cpu().numpy(), want_out), flags
 
 
 def test_wide_accumulators_merge_without_norms(hdqt):

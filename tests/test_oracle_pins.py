@@ -222,12 +222,22 @@ def test_sr_integers_never_move_and_top_saturates():
 
 
 def test_sr_probability_is_fraction_of_fixed_point_value():
-    """P(up) = frac(rint(v 2^16) / 2^16) exactly: count over ALL 2^16 values of the random half-word."""
-    for v in [0.3, -1.7, 2.000031]:
-        v32 = np.float32(v)
-        v_fx = int(np.rint(np.float64(v32) * 65536.0))
-        ups = sum(((v_fx + u) >> 16) - (v_fx >> 16) for u in range(0, 65536, 1))
-        assert ups == v_fx & 0xFFFF
+    """P(up) = frac(rint(v 2^16) / 2^16): the oracle's up-count over 2^17 independent draws of one value
+    against that probability (a wrong half-word, a shifted fraction or a biased draw fails the 4-sigma gate),
+    and the degenerate fractions 0 and 1 - 2^-16 exactly."""
+    n = 1 << 17
+    for j, v in enumerate([0.3, -1.7, 2.000031, 5.75, -0.0001]):
+        draws = _sr_draws([v], n, seed=99 + j)[v]
+        v_fx = int(np.rint(np.float64(np.float32(v)) * 65536.0))
+        p_up = (v_fx & 0xFFFF) / 65536.0
+        ups = int((draws - (v_fx >> 16)).sum())
+        assert set(np.unique(draws - (v_fx >> 16))) <= {0, 1}
+        assert abs(ups - n * p_up) <= 4.0 * np.sqrt(n * p_up * (1 - p_up)) + 1
+    # fraction exactly 0: never up; fraction 65535/65536: up unless the draw is 0 (expected ~2 misses in 2^17)
+    assert np.all(_sr_draws([3.0], 4096, seed=5)[3.0] == 3)
+    top = np.float32(2.0 + 65535.0 / 65536.0)
+    d = _sr_draws([float(top)], n, seed=6)[float(top)]
+    assert 0 <= int((d == 2).sum()) <= 12 and np.all((d == 2) | (d == 3))
 
 
 def test_sr_deterministic_and_seed_sensitive():
@@ -339,15 +349,59 @@ def test_calibrate_acc_shift():
 
 # ---------------------------------------------------------- end to end ------
 
-def test_three_gemms_shapes_and_operand_roles():
+# What the paper fixes per product (Section 3, sensitivity paragraph: stochastic rounding on the two gradient
+# operands and on the activation of the backward pass; Section 4: clip 0.975 on the forward operands), written
+# out once more here as literals and compared with the oracle's descriptor tables.
+ROLE_TABLE = {
+    #          round_a  round_b  clip_a  clip_b
+    "fwd":   (0,       0,       0.975,  0.975),    # X nearest, W nearest
+    "dgrad": (1,       0,       1.0,    1.0),      # G stochastic, W nearest
+    "wgrad": (1,       1,       1.0,    1.0),      # X stochastic, G stochastic
+}
+
+
+def test_role_tables_follow_the_paper():
+    for kind, make in (("fwd", O.fwd_desc), ("dgrad", O.dgrad_desc), ("wgrad", O.wgrad_desc)):
+        d = make()
+        assert (d.round_a, d.round_b, d.clip_a, d.clip_b) == ROLE_TABLE[kind], kind
+        assert (d.in_bits, d.acc_bits, d.acc_tile, d.acc_shift, d.had_block) == (4, 8, 32, 0, 32), kind
+    assert (O.ROUND_NEAREST, O.ROUND_STOCHASTIC) == (0, 1)
+
+
+def test_three_gemms_shapes_roles_and_behaviour():
+    """Shapes, which operand is transposed, and the behaviour each role implies: a nearest-rounded operand does
+    not depend on the seed, a stochastically rounded one does; the forward scale carries the 0.975 clip."""
     from paper_2310_03675_b200 import inputs
     X, W, G = inputs.single_layer(0)
-    f = O.gemm_fwd(X, W, O.fwd_desc())
-    d = O.gemm_dgrad(G, W, O.dgrad_desc())
-    w = O.gemm_wgrad(X, G, O.wgrad_desc())
+    runs = {}
+    for seed in (0, 1):
+        runs[seed] = (O.gemm_fwd(X, W, O.fwd_desc(seed=seed)), O.gemm_dgrad(G, W, O.dgrad_desc(seed=seed)),
+                      O.gemm_wgrad(X, G, O.wgrad_desc(seed=seed)))
+    f, d, w = runs[0]
     assert f["out"].shape == (32, 64) and f["Aq"].shape == (32, 128) and f["Bq"].shape == (64, 128)
     assert d["out"].shape == (32, 128) and d["Aq"].shape == (32, 64) and d["Bq"].shape == (128, 64)
     assert w["out"].shape == (128, 64) and w["Aq"].shape == (128, 32) and w["Bq"].shape == (64, 32)
+    # operands and their transposes: each code matrix equals the quantizer run on the stated view
+    for res, a_view, b_view in ((f, X, W.T), (d, G, W), (w, X.T, G.T)):
+        d0 = O.GemmDesc()
+        for name, view, rnd, clip, tag in (("Aq", a_view, res is not f, 0.975 if res is f else 1.0, d0.tag_a),
+                                           ("Bq", b_view, res is w, 0.975 if res is f else 1.0, d0.tag_b)):
+            want, _, _ = O.quantize_hadamard(np.ascontiguousarray(view), 32, 4, clip, int(rnd), seed=0, tag=tag)
+            assert np.array_equal(res[name], want), name
+    # seed dependence follows the rounding mode of each operand
+    f1, d1, w1 = runs[1]
+    assert np.array_equal(f["Aq"], f1["Aq"]) and np.array_equal(f["Bq"], f1["Bq"])          # fwd: both nearest
+    assert not np.array_equal(d["Aq"], d1["Aq"]) and np.array_equal(d["Bq"], d1["Bq"])      # dgrad: G stochastic
+    assert not np.array_equal(w["Aq"], w1["Aq"]) and not np.array_equal(w["Bq"], w1["Bq"])  # wgrad: both
+    # the forward scale is 0.975 * max|xH| / 8 (one fp32 multiply, then an exact power of two); backward: max / 8
+    xh = O.fwht_blockdiag(O.pad_contraction(X, 32), 32)
+    gh = O.fwht_blockdiag(O.pad_contraction(G, 32), 32)
+    amax_x, amax_g = np.float32(np.abs(xh).max()), np.float32(np.abs(gh).max())
+    assert f["step_a"] == np.float32(np.float32(0.975) * amax_x) * np.float32(0.125)
+    assert d["step_a"] == amax_g * np.float32(0.125)
+    # with the clip, every transformed element above 0.975 max saturates at +7 / -8 (Section 4)
+    v = xh / np.float32(np.float32(0.975) * amax_x) * 8
+    assert np.all(f["Aq"][v >= 7.5] == 7) and np.all(f["Aq"][v <= -8.0] == -8) and (v >= 7.5).any()
     # quantised results track the exact products (4-bit operands: loose bound)
     for res, exact in ((f, X @ W), (d, G @ W.T), (w, X.T @ G)):
         rel = np.linalg.norm(res["out"] - exact) / np.linalg.norm(exact)
