@@ -208,10 +208,10 @@ def test_runs_are_bitwise_reproducible(hdqt):
     assert not torch.equal(a, c)
 
 
-@pytest.mark.parametrize("size", [4096, 8192])
+@pytest.mark.parametrize("size", [4096, 8192, 16384])
 def test_sampled_parity_at_sweep_size(hdqt, size):
-    """Sweep-size dgrad-layout GEMM on heavy-tailed operands (8192 = the shape and launch configuration the
-    benchmark times): codes in full, outputs on sampled rows and columns."""
+    """Sweep-size dgrad-layout GEMM on heavy-tailed operands (16384 = the shape and launch configuration the
+    benchmark's headline times): codes in full, outputs on sampled rows and columns."""
     M = N = K = size
     A = inputs.heavy_tailed_torch(M, K, seed=100, device="cuda")
     B = inputs.heavy_tailed_torch(N, K, seed=101, device="cuda")
@@ -343,9 +343,10 @@ def test_wide_accumulators_merge_without_norms(hdqt):
         assert np.array_equal(S.cpu().numpy().astype(np.int64), plain)
 
 
-def test_sampled_parity_wgrad_layout_at_sweep_size(hdqt):
-    """4096^3 wgrad layout (both operands K-strided, both stochastic): codes in full, outputs sampled."""
-    M = N = K = 4096
+@pytest.mark.parametrize("size", [4096, 8192])
+def test_sampled_parity_wgrad_layout_at_sweep_size(hdqt, size):
+    """Sweep-size wgrad layout (both operands K-strided, both stochastic): codes in full, outputs sampled."""
+    M = N = K = size
     X = inputs.heavy_tailed_torch(K, M, seed=200, device="cuda")     # stored [Nb, D]: contraction index first
     G = inputs.heavy_tailed_torch(K, N, seed=201, device="cuda")
     desc = hdqt.default_desc("wgrad", seed=5)
