@@ -284,6 +284,36 @@ hdqt_status_t hdqt_gemm_wgrad(const hdqt_gemm_desc_t* desc /*host*/, const float
                               int32_t w_is_cd, void* workspace, size_t workspace_bytes,
                               int32_t* dev_status, void* stream);
 
+/*
+ * Convolution layers without a materialised im2col matrix (Section 3: the quantized matmul Z = X W is the
+ * product every layer lowers to; for a convolution X is the patch matrix of the input).  The transform and
+ * quantize kernels gather the patches straight from the NHWC activation tensor.
+ *
+ *   X : [batch, height, width, channels] fp32, contiguous, channels % 32 == 0 (else HDQT_ERR_UNSUPPORTED:
+ *       lower such a layer to hdqt_gemm_* on an explicit patch matrix)
+ *   W, dW : [Cout, kernel_h, kernel_w, channels] fp32, contiguous
+ *   Y, G  : [batch, Ho, Wo, Cout] fp32, contiguous, Ho = (height + 2 padding - kernel_h) / stride + 1
+ * The patch matrix has one row per output position (b, ho, wo) and its column index runs over
+ * (kh, kw, channel) with the channel fastest; padding pixels read as zero.  The results equal
+ * hdqt_gemm_fwd / hdqt_gemm_wgrad (w_is_cd = 1) on that matrix bit for bit; only hdqt_had_block = 32 is served.
+ * The data gradient of a convolution is hdqt_gemm_dgrad on G and W followed by the caller's scatter-add of the
+ * patch-matrix gradient (no implicit form is provided).
+ * Workspace: hdqt_workspace_bytes(desc, positions, Cout, kernel_h*kernel_w*channels) for the forward call,
+ * hdqt_workspace_bytes(desc, Cout, kernel_h*kernel_w*channels, positions) for the weight gradient.
+ */
+typedef struct hdqt_conv2d_geom {
+  int64_t batch, height, width, channels;
+  int32_t kernel_h, kernel_w, stride, padding;
+} hdqt_conv2d_geom_t;
+
+hdqt_status_t hdqt_conv2d_fwd(const hdqt_gemm_desc_t* desc /*host*/, const hdqt_conv2d_geom_t* geom /*host*/,
+                              const float* X, const float* W, float* Y, int64_t Cout, void* workspace,
+                              size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+hdqt_status_t hdqt_conv2d_wgrad(const hdqt_gemm_desc_t* desc /*host*/, const hdqt_conv2d_geom_t* geom /*host*/,
+                                const float* X, const float* G, float* dW, int64_t Cout, void* workspace,
+                                size_t workspace_bytes, int32_t* dev_status, void* stream);
+
 /* Workspace for any of the three calls on a GEMM of the given size
  * (codes of both operands, scales, tile norms, GEMM scratch). */
 size_t hdqt_workspace_bytes(const hdqt_gemm_desc_t* desc /*host*/, int64_t M, int64_t N,

@@ -27,6 +27,7 @@ constexpr int64_t kMinBlocksForNorms = 32;
 struct OperandView {  // logical [rows, K] view of an operand with the contraction index as "K"
   const float* src;
   int64_t rows, ld_row, ld_k;
+  ConvGeom conv{};    // enabled: src is an NHWC tensor and the view is its implicit im2col matrix (or its transpose)
 };
 
 }  // namespace
@@ -194,6 +195,7 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
   // argument rules of hdqt_quantize_hadamard, checked once for both operands
   if ((st = check_quant_args(gA.src, gA.rows, K, gA.ld_row, gA.ld_k, d->had_block)) != HDQT_OK) return st;
   if ((st = check_quant_args(gB.src, gB.rows, K, gB.ld_row, gB.ld_k, d->had_block)) != HDQT_OK) return st;
+  if ((gA.conv.enabled || gB.conv.enabled) && d->had_block != 32) return HDQT_ERR_UNSUPPORTED;
   if (d->in_bits < 2 || d->in_bits > 8) return HDQT_ERR_INVALID_ARG;
   if (!(clipA >= 1.0f / 64.0f && clipA <= 1.0f) || !(clipB >= 1.0f / 64.0f && clipB <= 1.0f))
     return HDQT_ERR_INVALID_ARG;
@@ -206,10 +208,10 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
   // both operands in one calibration and one quantize launch (per memory layout); measured maxima are
   // published where the layout says (harnesses read them back)
   QuantOperand ops[2];
-  ops[0] = QuantOperand{gA.src, gA.rows, K, gA.ld_row, gA.ld_k, clipA, roundA, tagA, amaxA,
+  ops[0] = QuantOperand{gA.src, gA.rows, K, gA.ld_row, gA.ld_k, gA.conv, clipA, roundA, tagA, amaxA,
                         reinterpret_cast<float*>(ws + L.amax_a), reinterpret_cast<int8_t*>(ws + L.codes_a),
                         reinterpret_cast<float*>(ws + L.step_a), normsA};
-  ops[1] = QuantOperand{gB.src, gB.rows, K, gB.ld_row, gB.ld_k, clipB, roundB, tagB, amaxB,
+  ops[1] = QuantOperand{gB.src, gB.rows, K, gB.ld_row, gB.ld_k, gB.conv, clipB, roundB, tagB, amaxB,
                         reinterpret_cast<float*>(ws + L.amax_b), reinterpret_cast<int8_t*>(ws + L.codes_b),
                         reinterpret_cast<float*>(ws + L.step_b), normsB};
   st = launch_calibrate_quantize(ops, 2, d->had_block, d->in_bits, d->seed,
@@ -254,4 +256,62 @@ extern "C" hdqt_status_t hdqt_gemm_wgrad(const hdqt_gemm_desc_t* d, const float*
   // dW[D,C] = (X^T)(G); for the [C,D] layout the operands trade places: dW^T[C,D] = (G^T)(X)
   if (w_is_cd) return run_gemm(d, a, b, true, Nb, dW, D, workspace, workspace_bytes, dev_status, stream);
   return run_gemm(d, a, b, false, Nb, dW, C, workspace, workspace_bytes, dev_status, stream);
+}
+
+// ---- convolution as an implicit im2col GEMM ----------------------------------------------------
+
+namespace {
+
+hdqt_status_t conv_geom(const hdqt_conv2d_geom_t* g, ConvGeom* out, int64_t* positions, int64_t* patch) {
+  if (!g || g->batch <= 0 || g->height <= 0 || g->width <= 0 || g->channels <= 0) return HDQT_ERR_INVALID_ARG;
+  if (g->kernel_h <= 0 || g->kernel_w <= 0 || g->stride <= 0 || g->padding < 0) return HDQT_ERR_INVALID_ARG;
+  if (g->channels % 32 != 0) return HDQT_ERR_UNSUPPORTED;     // a 32-wide K block must stay inside one input pixel
+  const int64_t Ho = (g->height + 2 * g->padding - g->kernel_h) / g->stride + 1;
+  const int64_t Wo = (g->width + 2 * g->padding - g->kernel_w) / g->stride + 1;
+  if (Ho <= 0 || Wo <= 0) return HDQT_ERR_INVALID_ARG;
+  const int64_t n = g->batch * Ho * Wo, k = (int64_t)g->kernel_h * g->kernel_w * g->channels;
+  if (n >= (int64_t(1) << 31) || k >= (int64_t(1) << 31) || g->height >= (1 << 30) || g->width >= (1 << 30))
+    return HDQT_ERR_UNSUPPORTED;
+  out->enabled = 1;
+  out->H = (int32_t)g->height; out->W = (int32_t)g->width; out->C = (int32_t)g->channels;
+  out->KW = g->kernel_w; out->stride = g->stride; out->pad = g->padding;
+  out->Ho = (int32_t)Ho; out->Wo = (int32_t)Wo;
+  out->div_c = make_fastdiv((uint32_t)g->channels);
+  out->div_kw = make_fastdiv((uint32_t)g->kernel_w);
+  out->div_wo = make_fastdiv((uint32_t)Wo);
+  out->div_ho = make_fastdiv((uint32_t)Ho);
+  *positions = n;
+  *patch = k;
+  return HDQT_OK;
+}
+
+}  // namespace
+
+extern "C" hdqt_status_t hdqt_conv2d_fwd(const hdqt_gemm_desc_t* d, const hdqt_conv2d_geom_t* g, const float* X,
+                                         const float* W, float* Y, int64_t Cout, void* workspace,
+                                         size_t workspace_bytes, int32_t* dev_status, void* stream) {
+  if (!X || !W || !Y || Cout <= 0) return HDQT_ERR_INVALID_ARG;
+  ConvGeom cg{};
+  int64_t n = 0, k = 0;
+  hdqt_status_t st = conv_geom(g, &cg, &n, &k);
+  if (st != HDQT_OK) return st;
+  // A = patches [positions, kh*kw*Cin] (contraction contiguous, gathered on the fly); B = W as [Cout, kh*kw*Cin]
+  OperandView a{X, n, k, 1, cg};
+  OperandView b{W, Cout, k, 1};
+  return run_gemm(d, a, b, false, k, Y, Cout, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" hdqt_status_t hdqt_conv2d_wgrad(const hdqt_gemm_desc_t* d, const hdqt_conv2d_geom_t* g, const float* X,
+                                           const float* G, float* dW, int64_t Cout, void* workspace,
+                                           size_t workspace_bytes, int32_t* dev_status, void* stream) {
+  if (!X || !G || !dW || Cout <= 0) return HDQT_ERR_INVALID_ARG;
+  ConvGeom cg{};
+  int64_t n = 0, k = 0;
+  hdqt_status_t st = conv_geom(g, &cg, &n, &k);
+  if (st != HDQT_OK) return st;
+  // contraction over the output positions: descriptor operand a = patches^T [kh*kw*Cin, positions], operand
+  // b = G^T [Cout, positions]; dW is written as [Cout, kh*kw*Cin], so the operands trade places in the GEMM
+  OperandView a{X, k, 1, k, cg};
+  OperandView b{G, Cout, 1, Cout};
+  return run_gemm(d, a, b, true, n, dW, k, workspace, workspace_bytes, dev_status, stream);
 }

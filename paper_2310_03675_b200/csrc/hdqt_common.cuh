@@ -87,10 +87,48 @@ inline hdqt_status_t cuda_failure(cudaError_t e, const char* what) {
 
 constexpr int kMaxPartials = 1024;   // partial calibration maxima per operand (>= thread blocks of a calibration launch)
 
-// One operand of a transform + quantize call: logical [rows, K], element (r, k) = src[r*ld_row + k*ld_k].
+// Implicit im2col view of an NHWC activation tensor x[B, H, W, C] (paper Section 3: the transform and the
+// quantizer act along the contraction dimension of the matmul a convolution lowers to): the logical matrix has
+// one row per output position (b, ho, wo) and the column index runs over (kh, kw, c) with c fastest; element
+// (n, k) is x[b, ho*stride + kh - pad, wo*stride + kw - pad, c], or 0 outside the image.  C must be a multiple
+// of 32, so that every 32-wide block of the column index is 32 consecutive channels of one input pixel.
+// Exact unsigned division by a run-time constant without a divide: q = (umulhi(n, m) + n) >> l with
+// l = ceil(log2 d), m = floor(2^32 (2^l - d) / d) + 1 (round-up method; exact for every n < 2^31, where the sum
+// cannot overflow).  The host fills m and l once per launch.
+struct FastDiv {
+  uint32_t d, m, l;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+  FastDiv f;
+  f.d = d;
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;
+  f.l = l;
+  f.m = (uint32_t)((((1ull << l) - d) << 32) / d + 1);
+  return f;
+}
+__device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv& f) { return (__umulhi(n, f.m) + n) >> f.l; }
+__device__ __forceinline__ void fastdivmod(uint32_t n, const FastDiv& f, uint32_t& q, uint32_t& r) {
+  q = fastdiv(n, f);
+  r = n - q * f.d;
+}
+
+struct ConvGeom {
+  int32_t enabled;        // 0 = plain matrix operand
+  int32_t H, W, C;        // input height, width, channels
+  int32_t KW;             // kernel width (the kernel height follows from the column count)
+  int32_t stride, pad;
+  int32_t Ho, Wo;         // output height, width
+  FastDiv div_c, div_kw, div_wo, div_ho;
+};
+
+// One operand of a transform + quantize call: logical [rows, K], element (r, k) = src[r*ld_row + k*ld_k]
+// (or the implicit im2col view above: ld_k == 1 then means "the contraction runs over the patch index", anything
+// else "the contraction runs over the output positions").
 struct QuantOperand {
   const float* src;
   int64_t rows, K, ld_row, ld_k;
+  ConvGeom conv;
   float clip;
   int32_t mode;          // hdqt_round_t
   uint32_t tag;

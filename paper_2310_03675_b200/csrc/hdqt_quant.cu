@@ -124,6 +124,65 @@ __device__ __forceinline__ void load8_kc(const float* __restrict__ row, int64_t 
   }
 }
 
+// ---- loads through the implicit im2col view ---------------------------------------------------
+
+// Address of the 8 consecutive patch elements k0..k0+7 of output position n (they lie inside one input pixel,
+// since C % 8 == 0), or nullptr if that pixel is padding.
+__device__ __forceinline__ const float* conv_chunk_ptr(const ConvGeom& g, const float* __restrict__ x, int64_t n,
+                                                       int64_t k0) {
+  uint32_t tap, c0, kh, kw, t, wo, b, ho;
+  fastdivmod((uint32_t)k0, g.div_c, tap, c0);
+  fastdivmod(tap, g.div_kw, kh, kw);
+  fastdivmod((uint32_t)n, g.div_wo, t, wo);
+  fastdivmod(t, g.div_ho, b, ho);
+  const int hi = (int)(ho * g.stride + kh) - g.pad, wi = (int)(wo * g.stride + kw) - g.pad;
+  if ((unsigned)hi >= (unsigned)g.H || (unsigned)wi >= (unsigned)g.W) return nullptr;
+  return x + (((int64_t)b * g.H + hi) * g.W + wi) * g.C + c0;
+}
+
+__device__ __forceinline__ void load8_conv(const ConvGeom& g, const float* __restrict__ x, int64_t n, int64_t k0,
+                                           bool vec, float (&v)[8]) {
+  const float* p = conv_chunk_ptr(g, x, n, k0);
+  if (p == nullptr) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = 0.0f;
+  } else if (vec) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(p + 4));
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __ldg(p + i);
+  }
+}
+
+// 32 consecutive output positions (32-block kb of the contraction) of patch element d: the positions are uniform
+// over the thread block and advance by one per element (no division inside the loop), the patch element
+// (tap, channel) is this thread's.
+__device__ __forceinline__ void load32_conv(const ConvGeom& g, const float* __restrict__ x, int64_t d, int64_t kb,
+                                            int64_t n_positions, float (&v)[32]) {
+  uint32_t tap, c, kh, kw, t, wo, b, ho;
+  fastdivmod((uint32_t)d, g.div_c, tap, c);
+  fastdivmod(tap, g.div_kw, kh, kw);
+  fastdivmod((uint32_t)(kb << 5), g.div_wo, t, wo);
+  fastdivmod(t, g.div_ho, b, ho);
+  const int dh = (int)kh - g.pad, dw = (int)kw - g.pad;
+  const int64_t left = n_positions - (kb << 5);
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    float val = 0.0f;
+    const int hi = (int)(ho * g.stride) + dh, wi = (int)(wo * g.stride) + dw;
+    if (i < left && (unsigned)hi < (unsigned)g.H && (unsigned)wi < (unsigned)g.W)
+      val = __ldg(x + (((int64_t)b * g.H + hi) * g.W + wi) * g.C + c);
+    v[i] = val;
+    if (++wo == (uint32_t)g.Wo) {
+      wo = 0;
+      if (++ho == (uint32_t)g.Ho) { ho = 0; ++b; }
+    }
+  }
+}
+
 // ---- quantizer --------------------------------------------------------------------------
 // Codes are produced with the offset 2^(bits-1) added (so that they are unsigned and one
 // min-with-relu instruction clamps both sides), packed four to a word, and the offset is taken out
@@ -235,6 +294,8 @@ struct QuantOp {
   uint32_t tag;
   int32_t vec;              // K contiguous: 128-bit loads allowed
   int32_t seg_log2;         // K contiguous, blocked mapping: log2 of the K segment a thread block covers
+  int32_t rt_log2;          // K strided: log2 of the rows a thread block covers (32..256; the rest of its 256
+                            // threads take further 32-blocks of K, so that operands with few rows fill the block)
   const float* amax_in;     // quantize: supplied maximum, or nullptr = reduce `partials`
   uint32_t* partials;       // calibration: one partial maximum (bit pattern) per thread block of this operand
   int32_t n_partials;
@@ -244,6 +305,7 @@ struct QuantOp {
   float* step_out;
   int32_t* tile_norms;
   int32_t first_block, num_blocks;
+  ConvGeom conv;            // enabled: src is an NHWC tensor viewed as its im2col matrix
 };
 
 struct QuantBatch {
@@ -346,7 +408,7 @@ absmax_kc_kernel(const __grid_constant__ QuantBatch b, int32_t* dev_status) {
   const int64_t chunks_per_row = op.K_pad >> 3;
   const int64_t total = op.rows * chunks_per_row;
   const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
-  const bool dense = (K == op.K_pad) && (ld_row == K);
+  const bool dense = (K == op.K_pad) && (ld_row == K) && !op.conv.enabled;
   const int lane = threadIdx.x & 31;
   uint32_t mx = 0u;
   for (int64_t base = (int64_t)local_block * (kThreads * kUnrollAbsmax); base < total;
@@ -361,7 +423,8 @@ absmax_kc_kernel(const __grid_constant__ QuantBatch b, int32_t* dev_status) {
         } else {
           int64_t r, k0;
           chunk_to_row_k(cmap, c, r, k0);
-          load8_kc(src + r * ld_row, k0, K, vec, x[u]);
+          if (op.conv.enabled) load8_conv(op.conv, src, r, k0, vec, x[u]);
+          else load8_kc(src + r * ld_row, k0, K, vec, x[u]);
         }
       } else {
 #pragma unroll
@@ -395,7 +458,7 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   const int64_t chunks_per_row = op.K_pad >> 3;
   const int64_t total = op.rows * chunks_per_row;
   const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
-  const bool dense = (K == op.K_pad) && (ld_row == K);
+  const bool dense = (K == op.K_pad) && (ld_row == K) && !op.conv.enabled;
   const int lane = threadIdx.x & 31;
   auto body = [&]<int kMode, bool kHad32>() {
   for (int64_t base = (int64_t)local_block * (kThreads * kUnrollQuant); base < total;
@@ -410,7 +473,8 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
         } else {
           int64_t r, k0;
           chunk_to_row_k(cmap, c, r, k0);
-          load8_kc(src + r * ld_row, k0, K, vec, x[u]);
+          if (op.conv.enabled) load8_conv(op.conv, src, r, k0, vec, x[u]);
+          else load8_kc(src + r * ld_row, k0, K, vec, x[u]);
         }
       } else {
 #pragma unroll
@@ -466,7 +530,7 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
     const bool k_ok = k0 < K_pad;
     int nmax = 0;
     const int64_t row0 = (rb << 7) + warp * rpw + row_sub;    // this thread's row in pass 0; a pass adds 8 * rpw rows
-    const bool whole = vec && ((rb << 7) + 128 <= rows) && (((kseg + 1) << op.seg_log2) <= K);
+    const bool whole = vec && !op.conv.enabled && ((rb << 7) + 128 <= rows) && (((kseg + 1) << op.seg_log2) <= K);
     if (whole) {
       // whole 128-row block, whole segment inside K, vector loads: nothing to test per chunk, running pointers
       const float* __restrict__ sp = src + row0 * ld_row + k0;
@@ -508,7 +572,8 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
         for (int u = 0; u < kUnrollQuant; ++u) {
           r[u] = row0 + (int64_t)(pass + u) * 8 * rpw;
           if (k_ok && r[u] < rows) {
-            load8_kc(src + r[u] * ld_row, k0, K, vec, x[u]);
+            if (op.conv.enabled) load8_conv(op.conv, src, r[u], k0, vec, x[u]);
+            else load8_kc(src + r[u] * ld_row, k0, K, vec, x[u]);
           } else {
             r[u] = -1;
 #pragma unroll
@@ -574,17 +639,23 @@ absmax_ks_kernel(const __grid_constant__ QuantBatch b, int32_t* dev_status) {
   const float* __restrict__ src = op.src;
   const int64_t rows = op.rows, K = op.K, ld_k = op.ld;
   const int had_block = b.had_block;
-  // work item = (32-block of K, group of kThreads rows); the host guarantees that their number fits 31 bits
-  const uint32_t row_groups = (uint32_t)((rows + kThreads - 1) / kThreads);
-  const uint32_t items = row_groups * (uint32_t)(op.K_pad >> 5);
+  // work item = (group of 2^rt_log2 rows, group of 256 >> rt_log2 32-blocks of K); the host guarantees that
+  // their number fits 31 bits
+  const int rt_log2 = op.rt_log2;
+  const int64_t T = op.K_pad >> 5;
+  const uint32_t row_groups = (uint32_t)((rows + (int64_t(1) << rt_log2) - 1) >> rt_log2);
+  const uint32_t kpc = (uint32_t)kThreads >> rt_log2;
+  const uint32_t items = row_groups * (uint32_t)((T + kpc - 1) / kpc);
+  const uint32_t r_local = threadIdx.x & ((1u << rt_log2) - 1u), kbs = threadIdx.x >> rt_log2;
   uint32_t mx = 0u;
   for (uint32_t w = (uint32_t)local_block; w < items; w += (uint32_t)op.num_blocks) {
-    const uint32_t kbu = w / row_groups;
-    const int64_t kb = kbu;
-    const int64_t r = (int64_t)(w - kbu * row_groups) * kThreads + threadIdx.x;
-    if (r < rows) {
+    const uint32_t kg = w / row_groups;
+    const int64_t kb = (int64_t)kg * kpc + kbs;
+    const int64_t r = ((int64_t)(w - kg * row_groups) << rt_log2) + r_local;
+    if (r < rows && kb < T) {
       float x[32];
-      load32_ks(src, r, kb, K, ld_k, x);
+      if (op.conv.enabled) load32_conv(op.conv, src, r, kb, K, x);
+      else load32_ks(src, r, kb, K, ld_k, x);
       fwht32_regs(x, had_block);
 #pragma unroll
       for (int i = 0; i < 32; ++i) mx = max(mx, abs_bits(x[i]));
@@ -609,19 +680,23 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   // rows are padded to a multiple of the block size so that one thread block never straddles
   // two 32-blocks of K and always covers whole 128-row groups (needed for the tile norms)
   const int64_t T = K_pad >> 5;
-  const uint32_t row_groups = (uint32_t)((rows + kThreads - 1) / kThreads);
-  const uint32_t items = row_groups * (uint32_t)T;   // the host guarantees that this fits 31 bits
+  const int rt_log2 = op.rt_log2;
+  const uint32_t row_groups = (uint32_t)((rows + (int64_t(1) << rt_log2) - 1) >> rt_log2);
+  const uint32_t kpc = (uint32_t)kThreads >> rt_log2;            // 32-blocks of K per work item
+  const uint32_t items = row_groups * (uint32_t)((T + kpc - 1) / kpc);   // the host guarantees that this fits 31 bits
+  const uint32_t r_local = threadIdx.x & ((1u << rt_log2) - 1u), kbs = threadIdx.x >> rt_log2;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   auto body = [&]<int kMode, bool kHad32>() {
   for (uint32_t item = (uint32_t)local_block; item < items; item += (uint32_t)op.num_blocks) {
-    const uint32_t kbu = item / row_groups;     // uniform over the block
-    const int64_t kb = kbu;
-    const int64_t r_group0 = (int64_t)(item - kbu * row_groups) * kThreads;
-    const int64_t r = r_group0 + threadIdx.x;
+    const uint32_t kg = item / row_groups;      // uniform over the block
+    const int64_t kb = (int64_t)kg * kpc + kbs;
+    const int64_t r_group0 = (int64_t)(item - kg * row_groups) << rt_log2;
+    const int64_t r = r_group0 + r_local;
     int ss = 0;
-    if (r < rows) {
+    if (r < rows && kb < T) {
       float x[32];
-      load32_ks(src, r, kb, K, ld_k, x);
+      if (op.conv.enabled) load32_conv(op.conv, src, r, kb, K, x);
+      else load32_ks(src, r, kb, K, ld_k, x);
       fwht32_regs<kHad32>(x, had_block);
       uint32_t w[8];
       const uint64_t g0 = (uint64_t)(r * K_pad + (kb << 5)) >> 3;
@@ -643,13 +718,16 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
       __syncthreads();
       if (lane == 0) s_norm[warp] = ss;
       __syncthreads();
-      if (threadIdx.x < kThreads / 128) {
-        const int64_t r_base = r_group0 + threadIdx.x * 128;
-        if (r_base < rows) {
+      // one writer per (128-row block, 32-block of K) pair of the item: its warps are consecutive
+      const uint32_t rb_per_item = max(1u, (1u << rt_log2) >> 7), wpp = min(4u, (1u << rt_log2) >> 5);
+      if (threadIdx.x < kpc * rb_per_item) {
+        const uint32_t pk = threadIdx.x / rb_per_item, prb = threadIdx.x - pk * rb_per_item;
+        const int64_t r_base = r_group0 + (int64_t)prb * 128, pkb = (int64_t)kg * kpc + pk;
+        if (r_base < rows && pkb < T) {
+          const uint32_t w0 = ((pk << rt_log2) + (prb << 7)) >> 5;
           int mx = 0;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) mx = max(mx, s_norm[threadIdx.x * 4 + i]);
-          tile_norms[(r_base >> 7) * T + kb] = mx;
+          for (uint32_t i = 0; i < wpp; ++i) mx = max(mx, s_norm[w0 + i]);
+          tile_norms[(r_base >> 7) * T + pkb] = mx;
         }
       }
     }
@@ -677,6 +755,12 @@ int pick_seg_log2(int64_t K_pad) {
   return 5;
 }
 
+// work items of the K-strided kernels: (group of 2^rt_log2 rows) x (group of 256 >> rt_log2 32-blocks of K)
+int64_t ks_items(int64_t rows, int64_t K_pad, int rt_log2) {
+  const int64_t rt = int64_t(1) << rt_log2, kpc = kThreads >> rt_log2;
+  return ((rows + rt - 1) / rt) * (((K_pad >> 5) + kpc - 1) / kpc);
+}
+
 QuantOp make_op(const QuantOperand& a, int32_t had_block, uint32_t* partials) {
   QuantOp o;
   o.src = a.src;
@@ -690,6 +774,8 @@ QuantOp make_op(const QuantOperand& a, int32_t had_block, uint32_t* partials) {
   o.tag = a.tag;
   o.vec = (kc && (a.ld_row % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0)) ? 1 : 0;
   o.seg_log2 = pick_seg_log2(o.K_pad);
+  o.rt_log2 = 8;
+  while (o.rt_log2 > 5 && (int64_t(1) << (o.rt_log2 - 1)) >= a.rows) --o.rt_log2;
   o.amax_in = a.amax_in;
   o.partials = partials;
   o.n_partials = 0;
@@ -700,6 +786,8 @@ QuantOp make_op(const QuantOperand& a, int32_t had_block, uint32_t* partials) {
   o.tile_norms = a.tile_norms;
   o.first_block = 0;
   o.num_blocks = 0;
+  o.conv = a.conv;
+  if (a.conv.enabled) o.vec = ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0) ? 1 : 0;
   return o;
 }
 
@@ -732,7 +820,7 @@ hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t l
     b.op[0].num_blocks = grid_for(rows * (b.op[0].K_pad >> 3), kThreads * kUnrollAbsmax, 4);
     absmax_kc_kernel<<<b.op[0].num_blocks, kThreads, 0, s>>>(b, dev_status);
   } else {
-    const int64_t items = ((rows + kThreads - 1) / kThreads) * (b.op[0].K_pad >> 5);
+    const int64_t items = ks_items(rows, b.op[0].K_pad, b.op[0].rt_log2);
     if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
     b.op[0].num_blocks = grid_for(items, 1, 3);
     absmax_ks_kernel<<<b.op[0].num_blocks, kThreads, 0, s>>>(b, dev_status);
@@ -747,7 +835,7 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
   for (int i = 0; i < n_ops; ++i) {
     op[i] = make_op(ops[i], had_block, partials + (size_t)i * kMaxPartials);
     if (ops[i].ld_k != 1) {
-      const int64_t items = ((ops[i].rows + kThreads - 1) / kThreads) * (op[i].K_pad >> 5);
+      const int64_t items = ks_items(ops[i].rows, op[i].K_pad, op[i].rt_log2);
       if (items >= (int64_t(1) << 31)) return HDQT_ERR_UNSUPPORTED;
     }
   }
@@ -763,7 +851,7 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
       if (layout == 0) {
         g = grid_for(op[i].rows * (op[i].K_pad >> 3), kThreads * kUnrollAbsmax, 4);
       } else {
-        g = grid_for(((op[i].rows + kThreads - 1) / kThreads) * (op[i].K_pad >> 5), 1, 3);
+        g = grid_for(ks_items(op[i].rows, op[i].K_pad, op[i].rt_log2), 1, 3);
       }
       op[i].n_partials = g;
       QuantOp& o = b.op[b.n_ops++];
@@ -794,7 +882,7 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
         const int64_t seg = int64_t(1) << op[i].seg_log2;
         g = grid_for(((op[i].rows + 127) / 128) * ((op[i].K_pad + seg - 1) / seg), 1, 4);
       } else {
-        g = grid_for(((op[i].rows + kThreads - 1) / kThreads) * (op[i].K_pad >> 5), 1, 3);
+        g = grid_for(ks_items(op[i].rows, op[i].K_pad, op[i].rt_log2), 1, 3);
       }
       QuantOp& o = b.op[b.n_ops++];
       o = op[i];

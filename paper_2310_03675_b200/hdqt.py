@@ -27,7 +27,7 @@ EXPORTED = [
     "hdqt_quantize_hadamard", "hdqt_quantize_workspace_bytes", "hdqt_gemm_i8_tiled",
     "hdqt_gemm_i8_workspace_bytes", "hdqt_calibrate_acc_shift", "hdqt_gemm_fwd", "hdqt_gemm_dgrad",
     "hdqt_gemm_wgrad", "hdqt_workspace_bytes", "hdqt_workspace_layout", "hdqt_quantize_hadamard_static",
-    "hdqt_selftest_bounded_wait",
+    "hdqt_selftest_bounded_wait", "hdqt_conv2d_fwd", "hdqt_conv2d_wgrad",
 ]
 
 
@@ -40,6 +40,12 @@ class GemmDesc(C.Structure):
         ("tag_a", C.c_uint32), ("tag_b", C.c_uint32), ("amax_a", C.c_void_p), ("amax_b", C.c_void_p),
         ("flags", C.c_uint32),
     ]
+
+
+class Conv2dGeom(C.Structure):
+    """Mirror of hdqt_conv2d_geom_t."""
+    _fields_ = [("batch", C.c_int64), ("height", C.c_int64), ("width", C.c_int64), ("channels", C.c_int64),
+                ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("stride", C.c_int32), ("padding", C.c_int32)]
 
 
 class WsLayout(C.Structure):
@@ -85,6 +91,9 @@ def _load() -> C.CDLL:
         getattr(lib, name).argtypes = [C.POINTER(GemmDesc), vp, vp, vp, i64, i64, i64, i32, vp, sz, vp, vp]
     lib.hdqt_selftest_bounded_wait.argtypes = [vp, vp, vp]
     lib.hdqt_selftest_bounded_wait.restype = C.c_int
+    for name in ("hdqt_conv2d_fwd", "hdqt_conv2d_wgrad"):
+        getattr(lib, name).argtypes = [C.POINTER(GemmDesc), C.POINTER(Conv2dGeom), vp, vp, vp, i64, vp, sz, vp, vp]
+        getattr(lib, name).restype = C.c_int
     lib.hdqt_workspace_bytes.argtypes = [C.POINTER(GemmDesc), i64, i64, i64]
     lib.hdqt_workspace_bytes.restype = sz
     lib.hdqt_workspace_layout.argtypes = [C.POINTER(GemmDesc), i64, i64, i64, C.POINTER(WsLayout)]
@@ -333,3 +342,53 @@ def gemm_wgrad(X, G, desc: Optional[GemmDesc] = None, w_is_cd: bool = False, wor
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=X.device)
     return _run("hdqt_gemm_wgrad", desc, X, G, out, Nb, D, Cg, w_is_cd, M, N, Nb, workspace, dev_status)
+
+
+# ---- convolution without a materialised patch matrix ------------------------------------------------
+
+def conv2d_out_size(H: int, W: int, kernel: int, stride: int, padding: int):
+    return (H + 2 * padding - kernel) // stride + 1, (W + 2 * padding - kernel) // stride + 1
+
+
+def conv2d_fwd(X, W, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc] = None, workspace=None,
+               dev_status=None, out=None):
+    """Y[B,Ho,Wo,Cout] from X[B,H,W,Cin] (NHWC, Cin % 32 == 0) and W[Cout,kh,kw,Cin]. Returns (Y, workspace)."""
+    _req(X, "X"); _req(W, "W")
+    desc = desc or default_desc("fwd")
+    B, H, Wd, Cin = X.shape
+    Cout, kh, kw, Cin2 = W.shape
+    if Cin2 != Cin:
+        raise ValueError("shape mismatch")
+    Ho, Wo = conv2d_out_size(H, Wd, kh, stride, padding)
+    g = Conv2dGeom(B, H, Wd, Cin, kh, kw, stride, padding)
+    M, N, K = B * Ho * Wo, Cout, kh * kw * Cin
+    if workspace is None:
+        workspace = Workspace(desc, M, N, K, X.device)
+    if out is None:
+        out = torch.empty((B, Ho, Wo, Cout), dtype=torch.float32, device=X.device)
+    _check(lib.hdqt_conv2d_fwd(C.byref(desc), C.byref(g), X.data_ptr(), W.data_ptr(), out.data_ptr(), Cout,
+                               workspace.buf.data_ptr(), workspace.buf.numel(), _ptr(dev_status), _stream()),
+           "hdqt_conv2d_fwd")
+    return out, workspace
+
+
+def conv2d_wgrad(X, G, kernel: int, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc] = None,
+                 workspace=None, dev_status=None, out=None):
+    """dW[Cout,kh,kw,Cin] from X[B,H,W,Cin] and G[B,Ho,Wo,Cout] (both NHWC). Returns (dW, workspace)."""
+    _req(X, "X"); _req(G, "G")
+    desc = desc or default_desc("wgrad")
+    B, H, Wd, Cin = X.shape
+    Cout = G.shape[3]
+    Ho, Wo = conv2d_out_size(H, Wd, kernel, stride, padding)
+    if tuple(G.shape[:3]) != (B, Ho, Wo):
+        raise ValueError("shape mismatch")
+    g = Conv2dGeom(B, H, Wd, Cin, kernel, kernel, stride, padding)
+    M, N, K = Cout, kernel * kernel * Cin, B * Ho * Wo
+    if workspace is None:
+        workspace = Workspace(desc, M, N, K, X.device)
+    if out is None:
+        out = torch.empty((Cout, kernel, kernel, Cin), dtype=torch.float32, device=X.device)
+    _check(lib.hdqt_conv2d_wgrad(C.byref(desc), C.byref(g), X.data_ptr(), G.data_ptr(), out.data_ptr(), Cout,
+                                 workspace.buf.data_ptr(), workspace.buf.numel(), _ptr(dev_status), _stream()),
+           "hdqt_conv2d_wgrad")
+    return out, workspace

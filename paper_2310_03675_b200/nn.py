@@ -176,29 +176,44 @@ def _weight_matrix(w):
 
 
 class HdqtConv2dFunction(torch.autograd.Function):
-    """y = conv2d(x, w) (no bias) with the forward, dX and dW products as HDQT GEMMs on the im2col matrix."""
+    """y = conv2d(x, w) (no bias) with the forward, dX and dW products as HDQT GEMMs on the patch (im2col)
+    matrix.  With cin % 32 == 0 the forward and dW products gather the patches straight from the NHWC
+    activation inside the library's transform/quantize kernels (no patch matrix is materialised); other layers
+    (the 3-channel stem) build the matrix with torch copies.  dX is the dgrad GEMM followed by the scatter-add
+    of the patch-matrix gradient."""
 
     @staticmethod
-    def forward(ctx, x, w, stride: int, padding: int, layer_id: int, seed: int, over: dict):
+    def forward(ctx, x, w, stride: int, padding: int, layer_id: int, seed: int, over: dict, implicit: bool):
         B, Cin, H, W = x.shape
         Cout, _, kh, kw = w.shape
-        xc, Ho, Wo = _im2col(x, kh, stride, padding)
-        wm = _weight_matrix(w).contiguous()
         d = _desc("fwd", layer_id, seed, **over)
-        y2d, _ = hdqt.gemm_fwd(xc, wm, desc=d, w_is_cd=True,
-                               workspace=_workspace(d, xc.shape[0], Cout, xc.shape[1], x.device))
-        ctx.save_for_backward(xc, wm)
-        ctx.meta = (layer_id, seed, over, (B, Cin, H, W), (Cout, Cin, kh, kw), stride, padding, Ho, Wo)
-        # [B*Ho*Wo, Cout] is the channels-last storage of [B, Cout, Ho, Wo]: no copy
-        return y2d.view(B, Ho, Wo, Cout).permute(0, 3, 1, 2)
+        implicit = implicit and Cin % 32 == 0 and d.had_block == 32
+        wk = w.permute(0, 2, 3, 1).contiguous()                   # [Cout, kh, kw, Cin]
+        wm = wk.view(Cout, kh * kw * Cin)
+        if implicit:
+            xn = _nhwc(x)
+            Ho, Wo = hdqt.conv2d_out_size(H, W, kh, stride, padding)
+            y4, _ = hdqt.conv2d_fwd(xn, wk, stride, padding, desc=d,
+                                    workspace=_workspace(d, B * Ho * Wo, Cout, kh * kw * Cin, x.device))
+            ctx.save_for_backward(xn, wm)
+        else:
+            xc, Ho, Wo = _im2col(x, kh, stride, padding)
+            y2d, _ = hdqt.gemm_fwd(xc, wm, desc=d, w_is_cd=True,
+                                   workspace=_workspace(d, xc.shape[0], Cout, xc.shape[1], x.device))
+            y4 = y2d.view(B, Ho, Wo, Cout)
+            ctx.save_for_backward(xc, wm)
+        ctx.meta = (layer_id, seed, over, (B, Cin, H, W), (Cout, Cin, kh, kw), stride, padding, Ho, Wo, implicit)
+        # [B, Ho, Wo, Cout] is the channels-last storage of [B, Cout, Ho, Wo]: no copy
+        return y4.permute(0, 3, 1, 2)
 
     @staticmethod
     def backward(ctx, g):
-        xc, wm = ctx.saved_tensors
-        layer_id, seed, over, xshape, wshape, stride, padding, Ho, Wo = ctx.meta
+        xs, wm = ctx.saved_tensors
+        layer_id, seed, over, xshape, wshape, stride, padding, Ho, Wo, implicit = ctx.meta
         B = xshape[0]
         Cout, Cin, kh, kw = wshape
-        g2d = _nhwc(g).view(B * Ho * Wo, Cout)
+        gn = _nhwc(g)                                             # [B, Ho, Wo, Cout]
+        g2d = gn.view(B * Ho * Wo, Cout)
         dx = dw = None
         if ctx.needs_input_grad[0]:
             d = _desc("dgrad", layer_id, seed, **over)
@@ -207,18 +222,24 @@ class HdqtConv2dFunction(torch.autograd.Function):
             dx = _col2im(dxc, xshape, kh, stride, padding, Ho, Wo)
         if ctx.needs_input_grad[1]:
             d = _desc("wgrad", layer_id, seed, **over)
-            dwm, _ = hdqt.gemm_wgrad(xc, g2d, desc=d, w_is_cd=True,
-                                     workspace=_workspace(d, Cout, wm.shape[1], xc.shape[0], g.device))
-            dw = dwm.view(Cout, kh, kw, Cin).permute(0, 3, 1, 2)
-        return dx, dw, None, None, None, None, None
+            if implicit:
+                dwk, _ = hdqt.conv2d_wgrad(xs, gn, kh, stride, padding, desc=d,
+                                           workspace=_workspace(d, Cout, wm.shape[1], g2d.shape[0], g.device))
+            else:
+                dwm, _ = hdqt.gemm_wgrad(xs, g2d, desc=d, w_is_cd=True,
+                                         workspace=_workspace(d, Cout, wm.shape[1], xs.shape[0], g.device))
+                dwk = dwm.view(Cout, kh, kw, Cin)
+            dw = dwk.permute(0, 3, 1, 2)
+        return dx, dw, None, None, None, None, None, None
 
 
 class HdqtConv2d(torch.nn.Module):
     """3x3 / 1x1 convolution without bias; quantized=False runs torch's fp32 convolution on the same weights."""
 
     def __init__(self, cin: int, cout: int, kernel: int, stride: int = 1, padding: int = 0, layer_id: int = 0,
-                 quantized: bool = True, **over):
+                 quantized: bool = True, implicit: bool = True, **over):
         super().__init__()
+        self.implicit = implicit     # False: always materialise the patch matrix
         self.weight = torch.nn.Parameter(torch.empty(cout, cin, kernel, kernel))
         torch.nn.init.kaiming_normal_(self.weight, mode="fan_out", nonlinearity="relu")
         self.stride, self.padding, self.layer_id, self.quantized, self.over = stride, padding, layer_id, quantized, over
@@ -227,7 +248,8 @@ class HdqtConv2d(torch.nn.Module):
     def forward(self, x):
         if not self.quantized:
             return torch.nn.functional.conv2d(x, self.weight, None, self.stride, self.padding)
-        return HdqtConv2dFunction.apply(x, self.weight, self.stride, self.padding, self.layer_id, self.step, self.over)
+        return HdqtConv2dFunction.apply(x, self.weight, self.stride, self.padding, self.layer_id, self.step, self.over,
+                                        self.implicit)
 
 
 class _BasicBlock(torch.nn.Module):

@@ -61,6 +61,15 @@ def test_conv_layer_matches_oracle_on_the_im2col_matrices(cin, cout, k, stride, 
     dxc = torch.from_numpy(want_dx["out"]).cuda()
     want_dx_img = hnn._col2im(dxc, x.shape, k, stride, pad, Ho, Wo)
     assert torch.equal(x.grad, want_dx_img)
+    # the same layer with the patch matrix materialised (no implicit gather) gives identical results
+    if cin % 32 == 0:
+        twin = hnn.HdqtConv2d(cin, cout, k, stride, pad, layer_id=3, implicit=False).cuda()
+        twin.load_state_dict(layer.state_dict())
+        twin.step = 11
+        x2 = x.detach().clone().requires_grad_(True)
+        y2 = twin(x2)
+        y2.backward(g)
+        assert torch.equal(y2, y) and torch.equal(x2.grad, x.grad) and torch.equal(twin.weight.grad, layer.weight.grad)
     # and the layer agrees with torch's fp32 convolution up to quantisation noise (layout / adjoint sanity)
     ref = torch.nn.functional.conv2d(x.detach(), layer.weight.detach(), None, stride, pad)
     rel = (y.detach() - ref).norm() / ref.norm()
