@@ -29,10 +29,10 @@ struct TileInfo {                       // what the certificate warp publishes p
 };
 static_assert(sizeof(TileInfo) == TILE_INFO_BYTES, "TileInfo layout");
 
+template <int GROUP_M = 16>
 __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tile_m, int& tile_n) {
   // grouped order: co-resident CTAs form a roughly square patch (16 row blocks x ~9 column blocks on
   // 148 SMs), so both operands' panels are shared through L2
-  constexpr int GROUP_M = 16;
   const int per_group = GROUP_M * tiles_n;
   const int group = t / per_group;
   const int first_m = group * GROUP_M;

@@ -16,6 +16,12 @@ namespace {
 // 128 x 256 blocks.  Two small kernels build the two work lists.
 
 constexpr int PAIR_M = 2 * BM;
+// Pair blocks are walked in groups of PAIR_GROUP_M block rows: the CTA pairs that run together then share few
+// enough operand panels (all of K) for the L2 to keep them between one wave of blocks and the next.
+#ifndef HDQT_PAIR_GROUP_M
+#define HDQT_PAIR_GROUP_M 16
+#endif
+constexpr int PAIR_GROUP_M = HDQT_PAIR_GROUP_M;
 
 // Class of pair block t (grouped order over [tiles_m2, tiles_n]) from the number u of its accumulator tiles
 // without a clamp-free certificate:  1 = none (pure),  2 = a few (u <= max_fix: the pair kernel accumulates them
@@ -43,7 +49,7 @@ __global__ void classify_pair_blocks_kernel(const int32_t* __restrict__ norms_a,
   const int lane = threadIdx.x & 31;
   if (t >= tiles_m2 * tiles_n) return;
   int tm, tn;
-  tile_coords(t, tiles_m2, tiles_n, tm, tn);
+  tile_coords<PAIR_GROUP_M>(t, tiles_m2, tiles_n, tm, tn);
   const int64_t T = tiles32;
   const int32_t* a0 = norms_a + (int64_t)(2 * tm) * T;
   const int32_t* b0 = norms_b + (int64_t)(2 * tn) * T;
@@ -74,7 +80,7 @@ compact_blocks_kernel(const uint8_t* __restrict__ flag, int tiles_m2, int tiles_
     const int t = base + threadIdx.x;
     int tm = 0, tn = 0, is_pair = 0, singles = 0, cls = 0;
     if (t < n) {
-      tile_coords(t, tiles_m2, tiles_n, tm, tn);
+      tile_coords<PAIR_GROUP_M>(t, tiles_m2, tiles_n, tm, tn);
       cls = flag[t];
       is_pair = (cls != 0);
       if (!is_pair) singles = ((int64_t)(2 * tm + 1) * 128 < M) ? 2 : 1;
@@ -225,7 +231,7 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   // i-th block of this launch; returns true if its sums are to be parked as integers for the fix-up pass
   auto block_at = [&](int i, int& tm, int& tn) {
     const int t = (p.block_list != nullptr) ? __ldg(p.block_list + i) : i;
-    tile_coords(t & ~kFixFlag, tiles_m2, tiles_n, tm, tn);
+    tile_coords<PAIR_GROUP_M>(t & ~kFixFlag, tiles_m2, tiles_n, tm, tn);
     return (t & kFixFlag) != 0;
   };
 
@@ -368,7 +374,7 @@ fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict
   const float scale = dequant_scale(p);
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
     int tm, tn;
-    tile_coords(__ldg(list_fix + item / (PAIR_M / FIX_ROWS)), tiles_m2, tiles_n, tm, tn);
+    tile_coords<PAIR_GROUP_M>(__ldg(list_fix + item / (PAIR_M / FIX_ROWS)), tiles_m2, tiles_n, tm, tn);
     const int64_t m0 = (int64_t)tm * PAIR_M + (item % (PAIR_M / FIX_ROWS)) * FIX_ROWS, n0 = (int64_t)tn * BN;
     if (m0 >= p.M) continue;     // block-uniform: these rows of a ragged last block do not exist
     // certificates are those of the whole pair block (what the pair kernel relied on)
