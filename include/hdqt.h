@@ -71,6 +71,7 @@ typedef enum {
 /* flags for the GEMM entry points */
 #define HDQT_FLAG_NO_MERGE 1u   /* never merge provably clamp-free tiles (see hdqt_gemm_i8_tiled) */
 #define HDQT_FLAG_NO_SPLIT_K 2u /* never cut a long contraction with few output blocks into several work items */
+#define HDQT_FLAG_RELU 4u       /* the three-GEMM / convolution calls: max(., 0) after the scale (and the bias)      */
 
 /*
  * Parameters of one HDQT GEMM Out[M,N] = A[M,K] B[K,N] (Section 3).
@@ -95,6 +96,10 @@ typedef struct hdqt_gemm_desc {
                           (skips the calibration pass); NULL = measure                 */
   const float* amax_b;
   uint32_t flags;     /* HDQT_FLAG_*                                                   */
+  const float* bias;  /* optional device fp32 [N], N = columns of the call's output: Out = fp32(S)*scale + bias[n],
+                         one fp32 multiply and one fp32 add per element, then the optional ReLU.  Bias and
+                         activation are outside the quantized path (Section 3 quantizes the matmul's inputs and
+                         accumulators only); fusing them saves the output's round trip.  NULL = none      */
 } hdqt_gemm_desc_t;
 
 /* Fills *d with the paper's defaults for kind 0 = forward, 1 = dgrad, 2 = wgrad

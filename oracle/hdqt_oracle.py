@@ -258,7 +258,7 @@ def num_tiles(K_pad: int, acc_tile: int) -> int:
 
 def gemm_i8_tiled(Aq: np.ndarray, Bq: np.ndarray, step_a, step_b,
                   acc_bits: int = 8, acc_tile: int = 32, acc_shift: int = 0,
-                  had_block: int = 32, want_tiles: bool = False):
+                  had_block: int = 32, want_tiles: bool = False, bias=None, relu: bool = False):
     """Out[M,N] from codes Aq[M,K_pad], Bq[N,K_pad] (both K contiguous).
 
     For every tile t of s consecutive k:   P_t = sum_k a[m,k] b[n,k]   (exact)
@@ -288,6 +288,12 @@ def gemm_i8_tiled(Aq: np.ndarray, Bq: np.ndarray, step_a, step_b,
     scale = F32(np.float64(F32(step_a)) * np.float64(F32(step_b))
                 * (2.0 ** int(acc_shift)) / float(had_block))
     out = (S.astype(F32) * scale).astype(F32)
+    # fp32 tail outside the quantized path (only the matmul's inputs and accumulators are quantized, Section 3):
+    # bias of the output column (one fp32 add), then ReLU
+    if bias is not None:
+        out = (out + np.asarray(bias, dtype=F32)[None, :]).astype(F32)
+    if relu:
+        out = np.maximum(out, F32(0.0))
     return out, S, tiles
 
 
@@ -303,12 +309,13 @@ class GemmDesc:
     def __init__(self, in_bits=4, acc_bits=8, acc_tile=32, acc_shift=0,
                  had_block=32, clip_a=1.0, clip_b=1.0,
                  round_a=ROUND_NEAREST, round_b=ROUND_NEAREST,
-                 seed=0, tag_a=0, tag_b=1):
+                 seed=0, tag_a=0, tag_b=1, bias=None, relu=False):
         self.in_bits, self.acc_bits, self.acc_tile = in_bits, acc_bits, acc_tile
         self.acc_shift, self.had_block = acc_shift, had_block
         self.clip_a, self.clip_b = clip_a, clip_b
         self.round_a, self.round_b = round_a, round_b
         self.seed, self.tag_a, self.tag_b = seed, tag_a, tag_b
+        self.bias, self.relu = bias, relu
 
 
 def hdqt_gemm(A_mk: np.ndarray, B_nk: np.ndarray, d: GemmDesc, want_tiles=False):
@@ -320,7 +327,7 @@ def hdqt_gemm(A_mk: np.ndarray, B_nk: np.ndarray, d: GemmDesc, want_tiles=False)
     Bq, sb, amax_b = quantize_hadamard(B_nk, d.had_block, d.in_bits, d.clip_b,
                                        d.round_b, d.seed, d.tag_b)
     out, S, tiles = gemm_i8_tiled(Aq, Bq, sa, sb, d.acc_bits, d.acc_tile,
-                                  d.acc_shift, d.had_block, want_tiles)
+                                  d.acc_shift, d.had_block, want_tiles, d.bias, d.relu)
     return dict(out=out, S=S, tiles=tiles, Aq=Aq, Bq=Bq, step_a=sa, step_b=sb,
                 amax_a=amax_a, amax_b=amax_b)
 

@@ -217,10 +217,10 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
   st = launch_calibrate_quantize(ops, 2, d->had_block, d->in_bits, d->seed,
                                  reinterpret_cast<uint32_t*>(ws + L.gemm_ws), dev_status, s);
   if (st != HDQT_OK) return st;
-  return hdqt_gemm_i8_tiled(reinterpret_cast<int8_t*>(ws + L.codes_a), reinterpret_cast<int8_t*>(ws + L.codes_b),
+  return gemm_i8_tiled_impl(reinterpret_cast<int8_t*>(ws + L.codes_a), reinterpret_cast<int8_t*>(ws + L.codes_b),
                             reinterpret_cast<float*>(ws + L.step_a), reinterpret_cast<float*>(ws + L.step_b), M, N,
                             L.k_pad, d->in_bits, d->acc_bits, d->acc_tile, d->acc_shift, d->had_block, out, ld_out, nullptr,
-                            nullptr, 0, normsA, normsB, d->flags, ws + L.gemm_ws, scratch_bytes, dev_status,
+                            nullptr, 0, normsA, normsB, d->flags, d->bias, ws + L.gemm_ws, scratch_bytes, dev_status,
                             stream);
 }
 

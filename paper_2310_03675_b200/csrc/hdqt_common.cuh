@@ -149,6 +149,14 @@ hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t l
 hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int32_t had_block, int32_t bits,
                                         uint64_t seed, uint32_t* partials, int32_t* dev_status, cudaStream_t s);
 
+// hdqt_gemm_i8_tiled plus an optional output-column bias (fp32 [N]); HDQT_FLAG_RELU in `flags` clamps at zero
+hdqt_status_t gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const float* step_a, const float* step_b,
+                                 int64_t M, int64_t N, int64_t K_pad, int32_t code_bits, int32_t acc_bits,
+                                 int32_t acc_tile, int32_t acc_shift, int32_t had_block, float* out, int64_t ld_out,
+                                 int32_t* S_out, void* tiles_out, int32_t tiles_elem_bytes, const int32_t* norms_a,
+                                 const int32_t* norms_b, uint32_t flags, const float* bias, void* workspace,
+                                 size_t workspace_bytes, int32_t* dev_status, void* stream);
+
 int sm_count();   // of the current device
 
 }  // namespace hdqt

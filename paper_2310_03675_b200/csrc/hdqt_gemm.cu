@@ -88,7 +88,7 @@ __global__ void split_k_finalize_kernel(const GemmParams p) {
     const int64_t m = i / p.N, n = i - m * p.N;
     float* o = p.out + m * p.ld_out + n;
     const int S = __float_as_int(*o);
-    *o = __fmul_rn((float)S, scale);
+    *o = finish1(p, __fmul_rn((float)S, scale), n);
     if (p.S_out != nullptr) p.S_out[i] = S;
   }
 }
@@ -176,6 +176,19 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
                                             const int32_t* norms_a, const int32_t* norms_b, uint32_t flags,
                                             void* workspace, size_t workspace_bytes, int32_t* dev_status,
                                             void* stream) {
+  return hdqt::gemm_i8_tiled_impl(Aq, Bq, step_a, step_b, M, N, K_pad, code_bits, acc_bits, acc_tile, acc_shift,
+                                  had_block, out, ld_out, S_out, tiles_out, tiles_elem_bytes, norms_a, norms_b, flags,
+                                  nullptr, workspace, workspace_bytes, dev_status, stream);
+}
+
+hdqt_status_t hdqt::gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const float* step_a,
+                                       const float* step_b, int64_t M, int64_t N, int64_t K_pad,
+                                       int32_t code_bits, int32_t acc_bits, int32_t acc_tile,
+                                       int32_t acc_shift, int32_t had_block, float* out, int64_t ld_out,
+                                       int32_t* S_out, void* tiles_out, int32_t tiles_elem_bytes,
+                                       const int32_t* norms_a, const int32_t* norms_b, uint32_t flags,
+                                       const float* bias, void* workspace, size_t workspace_bytes,
+                                       int32_t* dev_status, void* stream) {
   if (!Aq || !Bq || !step_a || !step_b || !out) return HDQT_ERR_INVALID_ARG;
   if (M <= 0 || N <= 0 || K_pad <= 0 || ld_out < N) return HDQT_ERR_INVALID_ARG;
   if (K_pad % 32 != 0) return HDQT_ERR_INVALID_ARG;
@@ -221,6 +234,8 @@ extern "C" hdqt_status_t hdqt_gemm_i8_tiled(const int8_t* Aq, const int8_t* Bq, 
   p.out = out; p.ld_out = ld_out; p.S_out = S_out;
   p.tiles_out = tiles_out; p.tiles_elem_bytes = tiles_elem_bytes;
   p.dev_status = dev_status;
+  p.bias = bias;
+  p.relu = (flags & HDQT_FLAG_RELU) ? 1 : 0;
 
   // 16-bit-lane epilogue: tile sums fit int16, the offset sums fit uint16 for flush_every tiles
   // (the epilogue forms P + 2^(b_a-1) in signed 16-bit lanes before it takes the minimum)

@@ -77,6 +77,8 @@ struct GemmParams {
   int32_t had_block;
   int32_t flush_every;    // packed mode: accumulator tiles summed in 16-bit lanes before widening
   int32_t offset_mma;     // packed mode: every clamp-path accumulator tile starts from the constant 2^(b_a-1)
+  const float* bias;      // optional fp32 [N]: added to the dequantised output (one fp32 add per element)
+  int32_t relu;           // != 0: max(., 0) after the bias
   int32_t split_k;        // > 1: the contraction of every output block is cut into this many work items
   int32_t split_kblocks;  // shared-memory stages (4 tiles of 32) per work item
   // merging of provably clamp-free accumulator tiles
@@ -354,6 +356,14 @@ __device__ __forceinline__ int acc_quant(int P, int r, int lo, int hi) {
   return min(max(P, lo), hi);
 }
 
+// The fp32 tail of the dequantising epilogue (outside the quantized path: Section 3 quantizes the matmul's inputs
+// and accumulators only): optional bias of the output column, optional ReLU.
+__device__ __forceinline__ float finish1(const GemmParams& p, float x, int64_t n) {
+  if (p.bias != nullptr) x = __fadd_rn(x, __ldg(p.bias + n));
+  if (p.relu) x = fmaxf(x, 0.0f);
+  return x;
+}
+
 // Writes 4 consecutive output columns of one row: the final fp32 values (and optionally the integer
 // sums), or - for an intermediate widening of the packed sums - the int32 partial sums, which are
 // parked in the output buffer itself until the final pass reads them back.
@@ -368,10 +378,10 @@ __device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t g
     }
     if (kFinal) {
       float4 o;
-      o.x = __fmul_rn((float)s[0], scale);
-      o.y = __fmul_rn((float)s[1], scale);
-      o.z = __fmul_rn((float)s[2], scale);
-      o.w = __fmul_rn((float)s[3], scale);
+      o.x = finish1(p, __fmul_rn((float)s[0], scale), gn);
+      o.y = finish1(p, __fmul_rn((float)s[1], scale), gn + 1);
+      o.z = finish1(p, __fmul_rn((float)s[2], scale), gn + 2);
+      o.w = finish1(p, __fmul_rn((float)s[3], scale), gn + 3);
       *reinterpret_cast<float4*>(orow) = o;
     } else {
       *reinterpret_cast<int4*>(orow) = make_int4(s[0], s[1], s[2], s[3]);
@@ -381,7 +391,7 @@ __device__ __forceinline__ void emit4(const GemmParams& p, int64_t gm, int64_t g
     for (int i = 0; i < 4; ++i) {
       if (gn + i < p.N) {
         if (have_prev) s[i] += __float_as_int(orow[i]);
-        orow[i] = kFinal ? __fmul_rn((float)s[i], scale) : __int_as_float(s[i]);
+        orow[i] = kFinal ? finish1(p, __fmul_rn((float)s[i], scale), gn + i) : __int_as_float(s[i]);
       }
     }
   }
@@ -466,7 +476,11 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
 #pragma unroll
     for (int rr = 0; rr < 32; rr += 8) {
       const int rloc = rr + sub;
-      const float4 v = *reinterpret_cast<const float4*>(e.box + rloc * 16 + ((quad + ((rloc >> 1) & 3)) & 3) * 4);
+      float4 v = *reinterpret_cast<const float4*>(e.box + rloc * 16 + ((quad + ((rloc >> 1) & 3)) & 3) * 4);
+      if (!raw && (p.bias != nullptr || p.relu)) {
+        const int64_t n = gn + quad * 4;
+        v.x = finish1(p, v.x, n); v.y = finish1(p, v.y, n + 1); v.z = finish1(p, v.z, n + 2); v.w = finish1(p, v.w, n + 3);
+      }
       const int64_t grow = (int64_t)job.m0 + e.q * 32 + rloc;
       if (grow < p.M) *reinterpret_cast<float4*>(p.out + grow * p.ld_out + gn + quad * 4) = v;
     }

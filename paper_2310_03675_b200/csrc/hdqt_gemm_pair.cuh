@@ -474,7 +474,7 @@ fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict
       for (int j = 0; j < 8; ++j) {
         const int64_t gn = n0 + lane + 32 * j;
         if (gm < p.M && gn < p.N) {
-          p.out[gm * p.ld_out + gn] = __fmul_rn((float)Sv[r][j], scale);
+          p.out[gm * p.ld_out + gn] = finish1(p, __fmul_rn((float)Sv[r][j], scale), gn);
           if (p.S_out != nullptr) p.S_out[gm * p.N + gn] = Sv[r][j];
         }
       }

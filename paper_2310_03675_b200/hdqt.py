@@ -18,6 +18,7 @@ ROUND_NEAREST = 0
 ROUND_STOCHASTIC = 1
 FLAG_NO_MERGE = 1
 FLAG_NO_SPLIT_K = 2
+FLAG_RELU = 4
 
 STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "WORKSPACE", "NONFINITE", "TIMEOUT", "CUDA",
                 "STATIC_SCRATCH"]
@@ -38,7 +39,7 @@ class GemmDesc(C.Structure):
         ("had_block", C.c_int32), ("clip_a", C.c_float), ("clip_b", C.c_float),
         ("round_a", C.c_int32), ("round_b", C.c_int32), ("seed", C.c_uint64),
         ("tag_a", C.c_uint32), ("tag_b", C.c_uint32), ("amax_a", C.c_void_p), ("amax_b", C.c_void_p),
-        ("flags", C.c_uint32),
+        ("flags", C.c_uint32), ("bias", C.c_void_p),
     ]
 
 
@@ -140,7 +141,7 @@ def default_desc(kind: str, **overrides) -> GemmDesc:
     d = GemmDesc()
     lib.hdqt_default_desc(C.byref(d), {"fwd": 0, "dgrad": 1, "wgrad": 2}[kind])
     for k, v in overrides.items():
-        if k in ("amax_a", "amax_b"):
+        if k in ("amax_a", "amax_b", "bias"):
             v = _ptr(v)
         setattr(d, k, v)
     return d

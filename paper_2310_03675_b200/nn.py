@@ -35,31 +35,41 @@ def _desc(kind: str, layer_id: int, seed: int, **over):
 
 
 class HdqtLinearFunction(torch.autograd.Function):
-    """y = x @ w with w stored [D, C]; forward, dX and dW are HDQT GEMMs."""
+    """y = act(x @ w + b) with w stored [D, C]; forward, dX and dW are HDQT GEMMs.  Bias and ReLU (both optional)
+    are applied inside the forward GEMM's dequantising epilogue."""
 
     @staticmethod
-    def forward(ctx, x, w, layer_id: int, seed: int, over: dict):
+    def forward(ctx, x, w, bias, relu: bool, layer_id: int, seed: int, over: dict):
         x = x.contiguous()
         w = w.contiguous()
-        d = _desc("fwd", layer_id, seed, **over)
+        extra = dict(over)
+        if bias is not None:
+            extra["bias"] = bias.contiguous()
+        if relu:
+            extra["flags"] = int(extra.get("flags", 0)) | hdqt.FLAG_RELU
+        d = _desc("fwd", layer_id, seed, **extra)
         y, _ = hdqt.gemm_fwd(x, w, desc=d, workspace=_workspace(d, x.shape[0], w.shape[1], x.shape[1], x.device))
-        ctx.save_for_backward(x, w)
-        ctx.meta = (layer_id, seed, over)
+        ctx.save_for_backward(x, w, y if relu else None)
+        ctx.meta = (layer_id, seed, over, bias is not None)
         return y
 
     @staticmethod
     def backward(ctx, g):
-        x, w = ctx.saved_tensors
-        layer_id, seed, over = ctx.meta
+        x, w, y = ctx.saved_tensors
+        layer_id, seed, over, has_bias = ctx.meta
         g = g.contiguous()
-        dx = dw = None
+        if y is not None:
+            g = g * (y > 0)
+        dx = dw = db = None
         if ctx.needs_input_grad[0]:
             d = _desc("dgrad", layer_id, seed, **over)
             dx, _ = hdqt.gemm_dgrad(g, w, desc=d, workspace=_workspace(d, g.shape[0], w.shape[0], g.shape[1], g.device))
         if ctx.needs_input_grad[1]:
             d = _desc("wgrad", layer_id, seed, **over)
             dw, _ = hdqt.gemm_wgrad(x, g, desc=d, workspace=_workspace(d, x.shape[1], g.shape[1], x.shape[0], x.device))
-        return dx, dw, None, None, None
+        if has_bias and ctx.needs_input_grad[2]:
+            db = g.sum(0)
+        return dx, dw, db, None, None, None, None
 
 
 class HdqtLinear(torch.nn.Module):
@@ -74,9 +84,8 @@ class HdqtLinear(torch.nn.Module):
         self.over = over
         self.step = 0          # advanced by the training loop; feeds the Philox seed
 
-    def forward(self, x):
-        y = HdqtLinearFunction.apply(x, self.weight, self.layer_id, self.step, self.over)
-        return y if self.bias is None else y + self.bias
+    def forward(self, x, relu: bool = False):
+        return HdqtLinearFunction.apply(x, self.weight, self.bias, relu, self.layer_id, self.step, self.over)
 
 
 class Mlp(torch.nn.Module):
@@ -95,9 +104,13 @@ class Mlp(torch.nn.Module):
 
     def forward(self, x):
         for i, l in enumerate(self.layers):
-            x = l(x) if self.quantized else x @ l.weight + l.bias
-            if i + 1 < len(self.layers):
-                x = torch.relu(x)
+            last = i + 1 == len(self.layers)
+            if self.quantized:
+                x = l(x, relu=not last)          # bias and ReLU inside the forward GEMM's epilogue
+            else:
+                x = x @ l.weight + l.bias
+                if not last:
+                    x = torch.relu(x)
         return x
 
 
@@ -305,10 +318,8 @@ class ResNet18Width(torch.nn.Module):
         n = head.weight.shape[1] if n_seen is None else n_seen
         w = head.weight if n == head.weight.shape[1] else head.weight[:, :n].contiguous()
         if self.quantized:
-            logits = HdqtLinearFunction.apply(y.contiguous(), w, head.layer_id, head.step, head.over)
-        else:
-            logits = y @ w
-        return logits + head.bias[:n]
+            return HdqtLinearFunction.apply(y.contiguous(), w, head.bias[:n], False, head.layer_id, head.step, head.over)
+        return y @ w + head.bias[:n]
 
 
 def class_patterns(classes: int, seed: int, device, size: int = 32, waves: int = 4):

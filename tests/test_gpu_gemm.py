@@ -563,3 +563,29 @@ def test_bounded_waits_run_out_and_report_timeout(hdqt):
     one = torch.ones(1, device="cuda")
     _, S, _ = hdqt.gemm_i8_tiled(_dev(A), _dev(A), one, one, want_S=True)
     assert (S == 32).all().item()
+
+
+@pytest.mark.parametrize("Nb,D,C,heavy", [(64, 96, 40, False), (300, 561, 130, False), (128 * 37 + 50, 1024, 256 * 33 + 24, True),
+                                          (70, 32 * 300, 50, False)])
+def test_fused_bias_and_relu(hdqt, Nb, D, C, heavy):
+    """Forward product with the bias and ReLU folded into the dequantising epilogue: small blocks, the work split of
+    large problems (pair kernel, fix-up pass, general kernel) and split-K all apply the same fp32 tail."""
+    if heavy:
+        X, W = inputs.heavy_tailed(Nb, D, seed=5), inputs.heavy_tailed(D, C, seed=6)
+    else:
+        X, W = inputs.activations(Nb, D, seed=Nb), inputs.weights(D, C, seed=C)
+    bias = inputs.activations(1, C, seed=7)[0] * np.float32(np.abs(X).mean() * np.abs(W).mean() * 4)
+    want = O.gemm_fwd(X, W, O.fwd_desc(tag_a=0, tag_b=1, bias=bias, relu=True))
+    status = hdqt.new_status("cuda")
+    bd = _dev(bias)
+    desc = hdqt.default_desc("fwd", bias=bd, flags=hdqt.FLAG_RELU)
+    out, ws = hdqt.gemm_fwd(_dev(X), _dev(W), desc=desc, dev_status=status)
+    hdqt.check_device_status(status)
+    assert np.array_equal(ws.codes_a().cpu().numpy(), want["Aq"])
+    got = out.cpu().numpy()
+    assert np.array_equal(got, want["out"])
+    assert (got == 0).mean() > 0.05 and (got > 0).mean() > 0.05      # the ReLU really cuts, the bias really shifts
+    # bias only
+    want_b = O.gemm_fwd(X, W, O.fwd_desc(tag_a=0, tag_b=1, bias=bias))
+    out_b, _ = hdqt.gemm_fwd(_dev(X), _dev(W), desc=hdqt.default_desc("fwd", bias=bd), dev_status=status)
+    assert np.array_equal(out_b.cpu().numpy(), want_b["out"])

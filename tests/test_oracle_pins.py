@@ -438,3 +438,23 @@ def test_sr_gemm_is_unbiased_on_average():
             errs.append(np.linalg.norm(acc / (seed + 1) - exact) / np.linalg.norm(exact))
     # 16x more samples -> about 4x less error; allow slack
     assert errs[1] < errs[0] / 2.5
+
+
+def test_bias_and_relu_tail_is_plain_fp32_arithmetic():
+    """The optional fp32 tail of the epilogue equals bias add and ReLU applied to the unfused result."""
+    rng = np.random.default_rng(21)
+    Aq = rng.integers(-8, 8, size=(9, 64)).astype(np.int8)
+    Bq = rng.integers(-8, 8, size=(5, 64)).astype(np.int8)
+    bias = rng.standard_normal(5).astype(np.float32)
+    plain, S, _ = O.gemm_i8_tiled(Aq, Bq, 0.01, 0.5)
+    fused, S2, _ = O.gemm_i8_tiled(Aq, Bq, 0.01, 0.5, bias=bias, relu=True)
+    assert np.array_equal(S, S2)
+    want = np.maximum((plain + bias[None, :]).astype(np.float32), np.float32(0))
+    assert np.array_equal(fused, want) and (fused == 0).any() and (fused > 0).any()
+    only_bias, _, _ = O.gemm_i8_tiled(Aq, Bq, 0.01, 0.5, bias=bias)
+    assert np.array_equal(only_bias, (plain + bias[None, :]).astype(np.float32))
+    X = rng.standard_normal((6, 40)).astype(np.float32)
+    W = rng.standard_normal((40, 5)).astype(np.float32)
+    a = O.gemm_fwd(X, W, O.fwd_desc())["out"]
+    b = O.gemm_fwd(X, W, O.fwd_desc(bias=bias, relu=True))["out"]
+    assert np.array_equal(b, np.maximum((a + bias).astype(np.float32), 0))
