@@ -354,7 +354,8 @@ def shape_record(case, steps, warmup, peaks):
 
 def train_steps_records(torch, dev, steps=20):
     """Training steps per second of the synthetic MLP and CNN workloads and of a class-incremental batch mix
-    (new-task samples + replayed exemplars, grown head), every matmul through the library; the fp32 torch step of
+    (new-task samples + replayed exemplars, grown head), every matmul through the library (with measured maxima,
+    and with delayed scaling: maxima carried from the previous step, no calibration pass); the fp32 torch step of
     the same model beside each.  Accuracy needs the long run (`--workload cil`)."""
     from paper_2310_03675_b200 import nn as hnn
     out = {}
@@ -373,9 +374,11 @@ def train_steps_records(torch, dev, steps=20):
 
     x, labels = hnn.sensor_window_batch(256, 1152, 12, seed=SEED, device=dev)
     rec = {}
-    for name, quantized in (("hdqt", True), ("fp32_torch", False)):
+    for name, quantized, over in (("hdqt", True, {}), ("hdqt_delayed_scaling", True, {"delayed": True}),
+                                  ("fp32_torch", False, {})):
         torch.manual_seed(0)
-        model = hnn.Mlp(quantized=quantized).to(dev)
+        hnn.reset_delayed_scaling()
+        model = hnn.Mlp(quantized=quantized, **over).to(dev)
         opt = torch.optim.SGD(model.parameters(), lr=0.01, momentum=0.9)
         ms = time_steps(lambda i: hnn.train_step(model, opt, x, labels, i), 5 * steps)
         rec[name] = {"steps_per_s": 1e3 / ms, "ms_per_step": ms}
@@ -387,9 +390,11 @@ def train_steps_records(torch, dev, steps=20):
     labels = torch.randint(0, 100, (128,), generator=g, device=dev)
     x = hnn.synthetic_images(labels, patterns, seed=SEED)
     rec = {}
-    for name, quantized in (("hdqt", True), ("fp32_torch", False)):
+    for name, quantized, over in (("hdqt", True, {}), ("hdqt_delayed_scaling", True, {"delayed": True}),
+                                  ("fp32_torch", False, {})):
         torch.manual_seed(0)
-        model = hnn.ResNet18Width(100, quantized=quantized).to(dev)
+        hnn.reset_delayed_scaling()
+        model = hnn.ResNet18Width(100, quantized=quantized, **over).to(dev)
         opt = torch.optim.SGD(model.parameters(), lr=0.05, momentum=0.9, weight_decay=2e-4)
         ms = time_steps(lambda i: hnn.cnn_train_step(model, opt, x, labels, i), steps)
         rec[name] = {"steps_per_s": 1e3 / ms, "ms_per_step": ms}
@@ -401,6 +406,7 @@ def train_steps_records(torch, dev, steps=20):
         out.setdefault("class_incremental_resnet18w_batch64new_64replay", {})[name] = \
             {"steps_per_s": 1e3 / ms, "ms_per_step": ms}
         del model, opt
+    hnn.reset_delayed_scaling()
     out["cnn_resnet18w_32x32_batch128"] = rec
     return out
 

@@ -100,7 +100,20 @@ typedef struct hdqt_gemm_desc {
                          one fp32 multiply and one fp32 add per element, then the optional ReLU.  Bias and
                          activation are outside the quantized path (Section 3 quantizes the matmul's inputs and
                          accumulators only); fusing them saves the output's round trip.  NULL = none      */
+  /* Delayed scaling (optional; Section 3 calibrates alpha from the tensor's maximum and leaves open when it
+     is measured).  amax_hist_out_*: device uint32[HDQT_AMAX_HISTORY_WORDS]; the call's quantize pass leaves the
+     partial maxima (fp32 bit patterns) of max|x H| of the operand it has just transformed there, at no extra
+     pass.  amax_hist_in_*: such an array from an EARLIER call (the same tensor one training step before); its
+     maximum replaces this call's calibration pass (4 of the 9 bytes per element), and values that have grown
+     beyond it saturate at the largest code.  amax_* (the scalar) takes precedence; in and out must be
+     different arrays.  NULL = not used.                                                                     */
+  const uint32_t* amax_hist_in_a;
+  const uint32_t* amax_hist_in_b;
+  uint32_t* amax_hist_out_a;
+  uint32_t* amax_hist_out_b;
 } hdqt_gemm_desc_t;
+
+#define HDQT_AMAX_HISTORY_WORDS 1024
 
 /* Fills *d with the paper's defaults for kind 0 = forward, 1 = dgrad, 2 = wgrad
  * (rounding modes and clip per Section 3 / Section 4). `d` is a host pointer. */

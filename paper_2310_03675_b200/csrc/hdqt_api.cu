@@ -208,10 +208,14 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
   // both operands in one calibration and one quantize launch (per memory layout); measured maxima are
   // published where the layout says (harnesses read them back)
   QuantOperand ops[2];
-  ops[0] = QuantOperand{gA.src, gA.rows, K, gA.ld_row, gA.ld_k, gA.conv, clipA, roundA, tagA, amaxA,
+  const uint32_t* histInA = swap ? d->amax_hist_in_b : d->amax_hist_in_a;
+  const uint32_t* histInB = swap ? d->amax_hist_in_a : d->amax_hist_in_b;
+  uint32_t* histOutA = swap ? d->amax_hist_out_b : d->amax_hist_out_a;
+  uint32_t* histOutB = swap ? d->amax_hist_out_a : d->amax_hist_out_b;
+  ops[0] = QuantOperand{gA.src, gA.rows, K, gA.ld_row, gA.ld_k, gA.conv, clipA, roundA, tagA, amaxA, histInA, histOutA,
                         reinterpret_cast<float*>(ws + L.amax_a), reinterpret_cast<int8_t*>(ws + L.codes_a),
                         reinterpret_cast<float*>(ws + L.step_a), normsA};
-  ops[1] = QuantOperand{gB.src, gB.rows, K, gB.ld_row, gB.ld_k, gB.conv, clipB, roundB, tagB, amaxB,
+  ops[1] = QuantOperand{gB.src, gB.rows, K, gB.ld_row, gB.ld_k, gB.conv, clipB, roundB, tagB, amaxB, histInB, histOutB,
                         reinterpret_cast<float*>(ws + L.amax_b), reinterpret_cast<int8_t*>(ws + L.codes_b),
                         reinterpret_cast<float*>(ws + L.step_b), normsB};
   st = launch_calibrate_quantize(ops, 2, d->had_block, d->in_bits, d->seed,

@@ -133,6 +133,8 @@ struct QuantOperand {
   int32_t mode;          // hdqt_round_t
   uint32_t tag;
   const float* amax_in;  // supplied calibration maximum (device) or nullptr = measure
+  const uint32_t* hist_in;  // or: kMaxPartials partial maxima left by an earlier call's quantize pass (delayed scaling)
+  uint32_t* hist_out;       // optional: this call's quantize pass leaves the partial maxima of ITS tensor here
   float* amax_slot;      // optional: where the measured maximum is published
   int8_t* codes;
   float* step_out;

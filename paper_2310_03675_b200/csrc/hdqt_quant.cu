@@ -249,18 +249,24 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams
 
 // Runs `body.template operator()<kMode, kHad32>()` for the operand's rounding mode and Hadamard block: the
 // per-chunk code is then free of mode and block-size tests (they cost more than a tenth of its instructions).
-template <typename Body>
-__device__ __forceinline__ void dispatch_mode(const QuantParams& p, int had_block, Body body) {
+template <bool kTrack, typename Body>
+__device__ __forceinline__ void dispatch_mode2(const QuantParams& p, int had_block, Body& body) {
   const int mode = (p.mode == HDQT_ROUND_NEAREST) ? 0 : (p.sr_magic ? 1 : 2);
   if (had_block == 32) {
-    if (mode == 0) body.template operator()<0, true>();
-    else if (mode == 1) body.template operator()<1, true>();
-    else body.template operator()<2, true>();
+    if (mode == 0) body.template operator()<0, true, kTrack>();
+    else if (mode == 1) body.template operator()<1, true, kTrack>();
+    else body.template operator()<2, true, kTrack>();
   } else {
-    if (mode == 0) body.template operator()<0, false>();
-    else if (mode == 1) body.template operator()<1, false>();
-    else body.template operator()<2, false>();
+    if (mode == 0) body.template operator()<0, false, kTrack>();
+    else if (mode == 1) body.template operator()<1, false, kTrack>();
+    else body.template operator()<2, false, kTrack>();
   }
+}
+// kTrack: the body also keeps the maximum magnitude of the transformed values it sees (delayed scaling)
+template <typename Body>
+__device__ __forceinline__ void dispatch_mode(const QuantParams& p, int had_block, bool track, Body body) {
+  if (track) dispatch_mode2<true>(p, had_block, body);
+  else dispatch_mode2<false>(p, had_block, body);
 }
 
 __device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bits, float clip, int mode,
@@ -299,6 +305,8 @@ struct QuantOp {
   const float* amax_in;     // quantize: supplied maximum, or nullptr = reduce `partials`
   uint32_t* partials;       // calibration: one partial maximum (bit pattern) per thread block of this operand
   int32_t n_partials;
+  const uint32_t* hist_in;  // quantize: kMaxPartials partial maxima of an earlier tensor, used when amax_in is null
+  uint32_t* hist_out;       // quantize: partial maxima of this tensor (kMaxPartials entries, unused ones zeroed)
   float* amax_atomic;       // calibration through the public call: atomic maximum into one float instead
   float* amax_slot;         // quantize: where the maximum that was used is published (may be null)
   int8_t* codes;
@@ -351,6 +359,20 @@ __device__ __forceinline__ void commit_partial_max(const QuantOp& op, int local_
   }
 }
 
+// Delayed scaling: the quantize pass leaves the partial maxima of the tensor it has just transformed, so that the
+// next call on the same tensor (the next training step) needs no calibration pass.  All kMaxPartials entries are
+// defined afterwards (the operand's first block zeroes the unused ones).
+__device__ __forceinline__ void commit_history(const QuantOp& op, int local_block, uint32_t mx, int32_t* dev_status) {
+  const uint32_t v = block_max_u32(mx);
+  if (threadIdx.x == 0) {
+    op.hist_out[local_block] = v;
+    if (v >= 0x7F800000u) report_status(dev_status, HDQT_ERR_NONFINITE);
+  }
+  if (local_block == 0) {
+    for (int i = op.num_blocks + threadIdx.x; i < kMaxPartials; i += kThreads) op.hist_out[i] = 0u;
+  }
+}
+
 // The calibration maximum a quantize block works with: the supplied one, or the maximum of the partial
 // maxima the calibration launch left behind.  Block 0 of the operand publishes scale and maximum.
 __device__ __forceinline__ QuantScale resolve_scale(const QuantOp& op, int local_block, int bits,
@@ -359,8 +381,11 @@ __device__ __forceinline__ QuantScale resolve_scale(const QuantOp& op, int local
   if (op.amax_in != nullptr) {
     amax = __ldg(op.amax_in);
   } else {
+    // partial maxima of this call's calibration pass, or those an earlier call's quantize pass left behind
+    const uint32_t* part = op.hist_in != nullptr ? op.hist_in : op.partials;
+    const int n = op.hist_in != nullptr ? kMaxPartials : op.n_partials;
     uint32_t mx = 0u;
-    for (int i = threadIdx.x; i < op.n_partials; i += kThreads) mx = max(mx, __ldcg(op.partials + i));
+    for (int i = threadIdx.x; i < n; i += kThreads) mx = max(mx, __ldcg(part + i));
     amax = __uint_as_float(block_max_u32(mx));
   }
   const QuantScale qs = make_quant_scale(amax, op.clip, bits);
@@ -460,7 +485,8 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   const ChunkMap cmap{chunks_per_row, total < (int64_t(1) << 31)};
   const bool dense = (K == op.K_pad) && (ld_row == K) && !op.conv.enabled;
   const int lane = threadIdx.x & 31;
-  auto body = [&]<int kMode, bool kHad32>() {
+  uint32_t seen = 0u;   // maximum |x H| this thread has seen (tracked only for delayed scaling)
+  auto body = [&]<int kMode, bool kHad32, bool kTrack>() {
   for (int64_t base = (int64_t)local_block * (kThreads * kUnrollQuant); base < total;
        base += (int64_t)op.num_blocks * (kThreads * kUnrollQuant)) {
     float x[kUnrollQuant][8];
@@ -486,6 +512,10 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
       const int64_t c = base + u * kThreads + threadIdx.x;
       fwht8_regs<kHad32>(x[u], had_block);
       fwht8_lanes<kHad32>(x[u], had_block, lane);
+      if (kTrack) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) seen = max(seen, abs_bits(x[u][i]));
+      }
       uint2 out;
       quantize8<kMode>(x[u], p, (uint64_t)c, out.x, out.y);  // linear index of the chunk's first element is 8*c
       // codes are dense [rows, K_pad]: chunk c is bytes [8c, 8c+8)
@@ -493,7 +523,8 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
     }
   }
   };
-  dispatch_mode(p, had_block, body);
+  dispatch_mode(p, had_block, op.hist_out != nullptr, body);
+  if (op.hist_out != nullptr) commit_history(op, local_block, seen, dev_status);
 }
 
 // quantize, blocked mapping, with the tile norms: a work item is 128 rows x one K segment of 2^seg_log2
@@ -523,7 +554,8 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
   const int64_t T = K_pad >> 5;
   const int64_t cpr = K_pad >> 3;                // chunks per code row
   const int64_t n_items = ((rows + 127) >> 7) * nseg;
-  auto body = [&]<int kMode, bool kHad32>() {
+  uint32_t seen = 0u;   // maximum |x H| this thread has seen (tracked only for delayed scaling)
+  auto body = [&]<int kMode, bool kHad32, bool kTrack>() {
   for (int64_t item = local_block; item < n_items; item += op.num_blocks) {
     const int64_t rb = item / nseg, kseg = item - rb * nseg;
     const int64_t k0 = (kseg << op.seg_log2) + (kc << 3);
@@ -551,6 +583,10 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
         for (int u = 0; u < kUnrollQuant; ++u) {
           fwht8_regs<kHad32>(x[u], had_block);
           fwht8_lanes<kHad32>(x[u], had_block, lane);
+          if (kTrack) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) seen = max(seen, abs_bits(x[u][i]));
+          }
           uint2 out;
           quantize8<kMode>(x[u], p, g + u * g_step, out.x, out.y);
           int ss = __dp4a((int)out.x, (int)out.x, 0);
@@ -584,6 +620,10 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
         for (int u = 0; u < kUnrollQuant; ++u) {
           fwht8_regs<kHad32>(x[u], had_block);
           fwht8_lanes<kHad32>(x[u], had_block, lane);
+          if (kTrack) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) seen = max(seen, abs_bits(x[u][i]));
+          }
           const bool valid = r[u] >= 0;
           const uint64_t g = valid ? (uint64_t)r[u] * (uint64_t)cpr + (uint64_t)(k0 >> 3) : 0u;
           uint2 out;
@@ -613,7 +653,8 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
     __syncthreads();
   }
   };
-  dispatch_mode(p, had_block, body);
+  dispatch_mode(p, had_block, op.hist_out != nullptr, body);
+  if (op.hist_out != nullptr) commit_history(op, local_block, seen, dev_status);
 }
 
 // ---- K-strided kernels ------------------------------------------------------------------------
@@ -686,7 +727,8 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   const uint32_t items = row_groups * (uint32_t)((T + kpc - 1) / kpc);   // the host guarantees that this fits 31 bits
   const uint32_t r_local = threadIdx.x & ((1u << rt_log2) - 1u), kbs = threadIdx.x >> rt_log2;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  auto body = [&]<int kMode, bool kHad32>() {
+  uint32_t seen = 0u;   // maximum |x H| this thread has seen (tracked only for delayed scaling)
+  auto body = [&]<int kMode, bool kHad32, bool kTrack>() {
   for (uint32_t item = (uint32_t)local_block; item < items; item += (uint32_t)op.num_blocks) {
     const uint32_t kg = item / row_groups;      // uniform over the block
     const int64_t kb = (int64_t)kg * kpc + kbs;
@@ -698,6 +740,10 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
       if (op.conv.enabled) load32_conv(op.conv, src, r, kb, K, x);
       else load32_ks(src, r, kb, K, ld_k, x);
       fwht32_regs<kHad32>(x, had_block);
+      if (kTrack) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) seen = max(seen, abs_bits(x[i]));
+      }
       uint32_t w[8];
       const uint64_t g0 = (uint64_t)(r * K_pad + (kb << 5)) >> 3;
 #pragma unroll
@@ -733,7 +779,8 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
     }
   }
   };
-  dispatch_mode(p, had_block, body);
+  dispatch_mode(p, had_block, op.hist_out != nullptr, body);
+  if (op.hist_out != nullptr) commit_history(op, local_block, seen, dev_status);
 }
 
 constexpr int kMaxDevices = 64;
@@ -779,6 +826,8 @@ QuantOp make_op(const QuantOperand& a, int32_t had_block, uint32_t* partials) {
   o.amax_in = a.amax_in;
   o.partials = partials;
   o.n_partials = 0;
+  o.hist_in = a.hist_in;
+  o.hist_out = a.hist_out;
   o.amax_atomic = nullptr;
   o.amax_slot = a.amax_slot;
   o.codes = a.codes;
@@ -846,7 +895,7 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
     b.bits = bits;
     int grid = 0;
     for (int i = 0; i < n_ops; ++i) {
-      if ((ops[i].ld_k != 1) != (layout == 1) || ops[i].amax_in != nullptr) continue;
+      if ((ops[i].ld_k != 1) != (layout == 1) || ops[i].amax_in != nullptr || ops[i].hist_in != nullptr) continue;
       int g;
       if (layout == 0) {
         g = grid_for(op[i].rows * (op[i].K_pad >> 3), kThreads * kUnrollAbsmax, 4);

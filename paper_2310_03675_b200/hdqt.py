@@ -19,6 +19,7 @@ ROUND_STOCHASTIC = 1
 FLAG_NO_MERGE = 1
 FLAG_NO_SPLIT_K = 2
 FLAG_RELU = 4
+AMAX_HISTORY_WORDS = 1024
 
 STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "WORKSPACE", "NONFINITE", "TIMEOUT", "CUDA",
                 "STATIC_SCRATCH"]
@@ -40,6 +41,8 @@ class GemmDesc(C.Structure):
         ("round_a", C.c_int32), ("round_b", C.c_int32), ("seed", C.c_uint64),
         ("tag_a", C.c_uint32), ("tag_b", C.c_uint32), ("amax_a", C.c_void_p), ("amax_b", C.c_void_p),
         ("flags", C.c_uint32), ("bias", C.c_void_p),
+        ("amax_hist_in_a", C.c_void_p), ("amax_hist_in_b", C.c_void_p),
+        ("amax_hist_out_a", C.c_void_p), ("amax_hist_out_b", C.c_void_p),
     ]
 
 
@@ -141,7 +144,7 @@ def default_desc(kind: str, **overrides) -> GemmDesc:
     d = GemmDesc()
     lib.hdqt_default_desc(C.byref(d), {"fwd": 0, "dgrad": 1, "wgrad": 2}[kind])
     for k, v in overrides.items():
-        if k in ("amax_a", "amax_b", "bias"):
+        if k in ("amax_a", "amax_b", "bias", "amax_hist_in_a", "amax_hist_in_b", "amax_hist_out_a", "amax_hist_out_b"):
             v = _ptr(v)
         setattr(d, k, v)
     return d

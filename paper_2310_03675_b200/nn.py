@@ -29,8 +29,37 @@ def _workspace(desc, M: int, N: int, K: int, device):
     return ws
 
 
-def _desc(kind: str, layer_id: int, seed: int, **over):
+# Delayed scaling (optional, `delayed=True` in the layer overrides): every (layer, product, operand) keeps two
+# history buffers of partial calibration maxima; a step quantizes with the maxima its predecessor left and leaves
+# its own (the library's quantize pass produces them for free), so that only a layer's first step runs the
+# calibration pass.
+_HISTORY = {}
+
+
+def _history(layer_id: int, kind: str, device):
+    key = (layer_id, kind, str(device))
+    h = _HISTORY.get(key)
+    if h is None:
+        h = _HISTORY[key] = {"bufs": [[torch.zeros(hdqt.AMAX_HISTORY_WORDS, dtype=torch.int32, device=device)
+                                       for _ in range(2)] for _ in range(2)], "calls": 0}
+    return h
+
+
+def reset_delayed_scaling():
+    """Forget every carried maximum (call when tensor shapes or roles change, e.g. between unrelated models)."""
+    _HISTORY.clear()
+
+
+def _desc(kind: str, layer_id: int, seed: int, device=None, **over):
     base = 8 * layer_id + 2 * _KIND[kind]
+    over = dict(over)
+    if over.pop("delayed", False) and device is not None:
+        h = _history(layer_id, kind, device)
+        cur, prev = h["bufs"][h["calls"] & 1], h["bufs"][(h["calls"] + 1) & 1]
+        over["amax_hist_out_a"], over["amax_hist_out_b"] = cur[0], cur[1]
+        if h["calls"] > 0:
+            over["amax_hist_in_a"], over["amax_hist_in_b"] = prev[0], prev[1]
+        h["calls"] += 1
     return hdqt.default_desc(kind, seed=seed, tag_a=base, tag_b=base + 1, **over)
 
 
@@ -47,7 +76,7 @@ class HdqtLinearFunction(torch.autograd.Function):
             extra["bias"] = bias.contiguous()
         if relu:
             extra["flags"] = int(extra.get("flags", 0)) | hdqt.FLAG_RELU
-        d = _desc("fwd", layer_id, seed, **extra)
+        d = _desc("fwd", layer_id, seed, x.device, **extra)
         y, _ = hdqt.gemm_fwd(x, w, desc=d, workspace=_workspace(d, x.shape[0], w.shape[1], x.shape[1], x.device))
         ctx.save_for_backward(x, w, y if relu else None)
         ctx.meta = (layer_id, seed, over, bias is not None)
@@ -62,10 +91,10 @@ class HdqtLinearFunction(torch.autograd.Function):
             g = g * (y > 0)
         dx = dw = db = None
         if ctx.needs_input_grad[0]:
-            d = _desc("dgrad", layer_id, seed, **over)
+            d = _desc("dgrad", layer_id, seed, g.device, **over)
             dx, _ = hdqt.gemm_dgrad(g, w, desc=d, workspace=_workspace(d, g.shape[0], w.shape[0], g.shape[1], g.device))
         if ctx.needs_input_grad[1]:
-            d = _desc("wgrad", layer_id, seed, **over)
+            d = _desc("wgrad", layer_id, seed, g.device, **over)
             dw, _ = hdqt.gemm_wgrad(x, g, desc=d, workspace=_workspace(d, x.shape[1], g.shape[1], x.shape[0], x.device))
         if has_bias and ctx.needs_input_grad[2]:
             db = g.sum(0)
@@ -199,7 +228,7 @@ class HdqtConv2dFunction(torch.autograd.Function):
     def forward(ctx, x, w, stride: int, padding: int, layer_id: int, seed: int, over: dict, implicit: bool):
         B, Cin, H, W = x.shape
         Cout, _, kh, kw = w.shape
-        d = _desc("fwd", layer_id, seed, **over)
+        d = _desc("fwd", layer_id, seed, x.device, **over)
         implicit = implicit and Cin % 32 == 0 and d.had_block == 32
         wk = w.permute(0, 2, 3, 1).contiguous()                   # [Cout, kh, kw, Cin]
         wm = wk.view(Cout, kh * kw * Cin)
@@ -229,12 +258,12 @@ class HdqtConv2dFunction(torch.autograd.Function):
         g2d = gn.view(B * Ho * Wo, Cout)
         dx = dw = None
         if ctx.needs_input_grad[0]:
-            d = _desc("dgrad", layer_id, seed, **over)
+            d = _desc("dgrad", layer_id, seed, g.device, **over)
             dxc, _ = hdqt.gemm_dgrad(g2d, wm, desc=d, w_is_cd=True,
                                      workspace=_workspace(d, g2d.shape[0], wm.shape[1], Cout, g.device))
             dx = _col2im(dxc, xshape, kh, stride, padding, Ho, Wo)
         if ctx.needs_input_grad[1]:
-            d = _desc("wgrad", layer_id, seed, **over)
+            d = _desc("wgrad", layer_id, seed, g.device, **over)
             if implicit:
                 dwk, _ = hdqt.conv2d_wgrad(xs, gn, kh, stride, padding, desc=d,
                                            workspace=_workspace(d, Cout, wm.shape[1], g2d.shape[0], g.device))

@@ -154,3 +154,56 @@ def test_tile_norms_of_wide_and_saturated_codes(hdqt, bits, clip):
             codes, _, norms = hdqt.quantize_hadamard(src, 32, bits, clip, 0, want_norms=True)
             assert np.array_equal(codes.cpu().numpy(), want_codes)
             assert np.array_equal(norms.cpu().numpy().astype(np.int64), _expected_norms(want_codes))
+
+
+@pytest.mark.parametrize("kind", ["dgrad", "wgrad", "fwd"])
+def test_delayed_scaling_uses_the_previous_tensors_maximum(hdqt, kind):
+    """Step 1 measures its maxima and leaves their partial maxima behind; step 2 quantizes DIFFERENT tensors with
+    step 1's maxima (no calibration pass) and leaves its own.  Codes, scales and outputs against the oracle run with
+    the same maxima; the history always holds exactly the maximum of the tensor just transformed."""
+    Nb, D, C = 300, 160, 200
+    X1, W1, G1 = inputs.single_layer(3, Nb=Nb, D=D, C=C)
+    X2, W2, G2 = inputs.single_layer(4, Nb=Nb, D=D, C=C)
+    X2, G2 = X2 * np.float32(1.7), G2 * np.float32(0.4)       # one operand grows (saturates), one shrinks
+    make = {"dgrad": (hdqt.gemm_dgrad, O.dgrad_desc, lambda X, W, G: (G, W), lambda X, W, G: (G, W)),
+            "wgrad": (hdqt.gemm_wgrad, O.wgrad_desc, lambda X, W, G: (X, G), lambda X, W, G: (X.T, G.T)),
+            "fwd": (hdqt.gemm_fwd, O.fwd_desc, lambda X, W, G: (X, W), lambda X, W, G: (X, W.T))}[kind]
+    call, odesc, pick, views = make
+    d0 = hdqt.default_desc(kind)
+    od = odesc(tag_a=d0.tag_a, tag_b=d0.tag_b, seed=3)
+    hist = [[torch.full((hdqt.AMAX_HISTORY_WORDS,), 0xFFFFFFFF, dtype=torch.int64, device="cuda").to(torch.int32)
+             for _ in range(2)] for _ in range(2)]          # [step parity][operand], pre-filled with garbage
+    status = hdqt.new_status("cuda")
+
+    def amax_h(v):
+        return np.float32(np.abs(O.fwht_blockdiag(O.pad_contraction(np.ascontiguousarray(v), 32), 32)).max())
+
+    def hist_max(t):
+        return float(t.view(torch.float32).max().item())
+
+    # step 1: measured maxima, history written
+    a1, b1 = pick(X1, W1, G1)
+    desc = hdqt.default_desc(kind, seed=3, amax_hist_out_a=hist[0][0], amax_hist_out_b=hist[0][1])
+    out1, ws = call(_dev(a1), _dev(b1), desc=desc, dev_status=status)
+    hdqt.check_device_status(status)
+    va, vb = views(X1, W1, G1)
+    want1 = O.hdqt_gemm(np.ascontiguousarray(va), np.ascontiguousarray(vb), od)
+    assert np.array_equal(out1.cpu().numpy(), want1["out"])
+    assert hist_max(hist[0][0]) == float(amax_h(va)) and hist_max(hist[0][1]) == float(amax_h(vb))
+    assert (hist[0][0] >= 0).all().item()                     # every entry defined: no garbage left (sign bit clear)
+    # step 2: other tensors, step 1's maxima, new history
+    a2, b2 = pick(X2, W2, G2)
+    desc = hdqt.default_desc(kind, seed=3, amax_hist_in_a=hist[0][0], amax_hist_in_b=hist[0][1],
+                             amax_hist_out_a=hist[1][0], amax_hist_out_b=hist[1][1])
+    out2, ws = call(_dev(a2), _dev(b2), desc=desc, dev_status=status)
+    hdqt.check_device_status(status)
+    va2, vb2 = views(X2, W2, G2)
+    Aq, sa, _ = O.quantize_hadamard(np.ascontiguousarray(va2), 32, 4, od.clip_a, od.round_a, 3, od.tag_a, amax=amax_h(va))
+    Bq, sb, _ = O.quantize_hadamard(np.ascontiguousarray(vb2), 32, 4, od.clip_b, od.round_b, 3, od.tag_b, amax=amax_h(vb))
+    assert np.array_equal(ws.codes_a().cpu().numpy(), Aq) and np.array_equal(ws.codes_b().cpu().numpy(), Bq)
+    assert ws.scalar("step_a").item() == float(sa) and ws.scalar("step_b").item() == float(sb)
+    want2, _, _ = O.gemm_i8_tiled(Aq, Bq, sa, sb)
+    assert np.array_equal(out2.cpu().numpy(), want2)
+    assert hist_max(hist[1][0]) == float(amax_h(va2)) and hist_max(hist[1][1]) == float(amax_h(vb2))
+    fresh, _, _ = O.quantize_hadamard(np.ascontiguousarray(va2), 32, 4, od.clip_a, od.round_a, 3, od.tag_a)
+    assert not np.array_equal(fresh, Aq)                       # the carried scale really differs from a fresh one
