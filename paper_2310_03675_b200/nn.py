@@ -388,11 +388,12 @@ def cnn_train_step(model: ResNet18Width, opt, x, labels, step: int, n_seen: Opti
 
 def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_task: int = 20,
                           steps_per_task: int = 1000, batch: int = 128, memory: int = 2000, seed: int = 0,
-                          lr: float = 0.05, test_per_class: int = 20, log=None, **over):
+                          lr: float = 0.05, test_per_class: int = 20, blend: float = 0.2, log=None, **over):
     """Plain-replay class-incremental training of the ResNet-18-width model on synthetic classes (paper
     Section 4: tasks arrive one after the other, a bounded memory of exemplars is replayed, the head grows with
     the classes seen; appendix: SGD lr 0.05, momentum 0.9, weight decay 2e-4, memory 2000).  Each batch mixes
-    new-task samples and replayed exemplars 1:1.  Returns a dict with the final accuracy over all classes seen,
+    new-task samples and replayed exemplars 1:1.  `blend` is the weight of the class pattern in an image (the rest
+    is uniform noise): small enough that the task is not solved trivially.  Returns a dict with the final accuracy over all classes seen,
     the accuracy after each task and the number of steps taken."""
     n_classes = tasks * classes_per_task
     patterns = class_patterns(n_classes, seed, device)
@@ -405,14 +406,14 @@ def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_t
     step = 0
     acc_after = []
     test_y = torch.arange(n_classes, device=device).repeat_interleave(test_per_class)
-    test_x = synthetic_images(test_y, patterns, seed=seed + 777)
+    test_x = synthetic_images(test_y, patterns, seed=seed + 777, blend=blend)
     for task in range(tasks):
         lo, hi = task * classes_per_task, (task + 1) * classes_per_task
         n_new = batch if mem_x is None else batch // 2
         model.train()
         for _ in range(steps_per_task):
             y = torch.randint(lo, hi, (n_new,), generator=g, device=device)
-            x = synthetic_images(y, patterns, seed=seed + 1000 + step)
+            x = synthetic_images(y, patterns, seed=seed + 1000 + step, blend=blend)
             if mem_x is not None:
                 idx = torch.randint(0, mem_x.shape[0], (batch - n_new,), generator=g, device=device)
                 x = torch.cat([x, mem_x[idx]])
@@ -427,7 +428,7 @@ def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_t
                 sel = (mem_y == c).nonzero().flatten()[:quota]
                 keep_x.append(mem_x[sel]); keep_y.append(mem_y[sel])
         new_y = torch.arange(lo, hi, device=device).repeat_interleave(quota)
-        keep_x.append(synthetic_images(new_y, patterns, seed=seed + 5000 + task)); keep_y.append(new_y)
+        keep_x.append(synthetic_images(new_y, patterns, seed=seed + 5000 + task, blend=blend)); keep_y.append(new_y)
         mem_x, mem_y = torch.cat(keep_x), torch.cat(keep_y)
         # accuracy over every class seen so far
         model.eval()
@@ -440,5 +441,5 @@ def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_t
             acc = float((torch.cat(pred) == test_y[m]).float().mean())
         acc_after.append(acc)
         if log:
-            log(f"task {task}: loss {float(loss):.3f} accuracy over {hi} classes {acc:.3f}")
+            log(f"task {task}: loss {loss.item():.3f} accuracy over {hi} classes {acc:.3f}")
     return {"final_accuracy": acc_after[-1], "accuracy_after_task": acc_after, "steps": step}
