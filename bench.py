@@ -486,6 +486,8 @@ def run_hdqt(args):
 
     elapsed_ms, quant_ms, gemm_ms = max_over_ranks([elapsed_ms, quant_ms, gemm_ms], dev, world)
     certified = case.certified_fraction() if rank == 0 else None
+    # in-run yardstick: MMA-only loop of the GEMM's instruction shape on every SM (no loads, no epilogue)
+    mma_probe_tops = hdqt.mma_rate_tops(dev_status=case.status) if rank == 0 else None
 
     sustained = clamp = supplied = None
     sweep, training = [], None
@@ -546,6 +548,8 @@ def run_hdqt(args):
             "roofline": {"bound": "tensor", "kernel": "hdqt_gemm_i8_tiled (pair kernel + fix-up + general kernel)",
                          "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak,
                          "peak_source": peak_src, "frac_of_datasheet_dense_int8": gemm_tops / DATASHEET_INT8_TOPS,
+                         "mma_only_probe_tops": mma_probe_tops,
+                         "frac_of_mma_only_probe": (gemm_tops / mma_probe_tops) if mma_probe_tops else None,
                          "traffic": None,
                          "traffic_note": "DRAM bytes of the GEMM kernels are captured with ncu on smaller shapes "
                                          "and do not scale linearly with the shape; they are listed per shape in "

@@ -275,6 +275,15 @@ hdqt_status_t hdqt_calibrate_acc_shift(const int8_t* Aq, const int8_t* Bq, int64
  */
 hdqt_status_t hdqt_selftest_bounded_wait(int32_t* dev_status, int32_t* gave_up, void* stream);
 
+/*
+ * Yardstick for the tiled matmul of Section 3 on this chip: every SM issues `iters` back-to-back
+ * tcgen05.mma.kind::i8 operations of the shape the GEMM kernels use (M128 N256 K32) on operands resident in
+ * shared memory - no loads, no epilogue.  The caller times the call with events; *ops_out (host, optional)
+ * receives the integer operations of the launch (2*128*256*32 per MMA and SM), so that ops / time is the
+ * integer tensor rate reached at the current clocks.
+ */
+hdqt_status_t hdqt_selftest_mma_rate(int32_t iters, int64_t* ops_out /*host*/, int32_t* dev_status, void* stream);
+
 /* ------------------------------------------------------------------------ */
 /* The three training GEMMs of one linear layer (Section 3: Z = X W and the    */
 /* backward products; X [Nb, D] activations, W weights, G = dL/dY [Nb, C])     */

@@ -80,6 +80,53 @@ __global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(int32_t* dev_
   if (threadIdx.x == 0 && abort_flag) report_status(dev_status, HDQT_ERR_TIMEOUT);
 }
 
+// ---- tensor-pipe yardstick: back-to-back MMAs of the shape the GEMM kernels use, operands resident ----
+// One CTA per SM, one thread issues `iters` tcgen05.mma.kind::i8 M128 N256 K32 into one accumulator from four
+// K slices of a zero-filled shared-memory stage; no loads, no epilogue.  Timed by the caller, it gives the
+// integer tensor rate this chip reaches at its current clocks: the ceiling the GEMM kernels are compared with.
+__global__ void __launch_bounds__(128, 1) mma_rate_kernel(int iters, int32_t* dev_status) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  const uint32_t base = smem_u32(smem_raw);
+  if (base & 1023u) {
+    if (threadIdx.x == 0) report_status(dev_status, HDQT_ERR_CUDA);
+    return;
+  }
+  for (int i = threadIdx.x; i < STAGE_BYTES / 16; i += blockDim.x) reinterpret_cast<uint4*>(smem_raw)[i] = make_uint4(0u, 0u, 0u, 0u);
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (threadIdx.x < 32) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(BN)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;
+  if (threadIdx.x == 32) {
+    const uint64_t da = make_smem_desc(base), db = make_smem_desc(base + A_STAGE);
+    for (int it = 0; it < iters; ++it) {
+      const uint64_t k = (uint64_t)(2 * (it & 3));
+      tc_mma_i8(tmem, da + k, db + k, it > 0 ? 1u : 0u);
+    }
+    tc_commit(smem_u32(&bar));
+    if (!mbar_wait(smem_u32(&bar), 0u, &abort_flag)) report_status(dev_status, HDQT_ERR_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(BN) : "memory");
+  }
+}
+
 // ---- split-K: integer sums parked in the output buffer -> fp32 result (and optional integer output) ----
 __global__ void split_k_finalize_kernel(const GemmParams p) {
   const float scale = dequant_scale(p);
@@ -381,3 +428,14 @@ extern "C" int hdqt_debug_timeline(long long* host_out) {
   return (int)cudaMemcpyFromSymbol(host_out, g_timeline, sizeof(long long) * 64 * 16);
 }
 #endif
+
+extern "C" hdqt_status_t hdqt_selftest_mma_rate(int32_t iters, int64_t* ops_out, int32_t* dev_status, void* stream) {
+  if (iters <= 0 || iters > (1 << 22)) return HDQT_ERR_INVALID_ARG;
+  cudaError_t e = cudaFuncSetAttribute(mma_rate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, STAGE_BYTES);
+  if (e != cudaSuccess) return cuda_failure(e, "cudaFuncSetAttribute(mma rate)");
+  const int sms = sm_count();
+  mma_rate_kernel<<<sms, 128, STAGE_BYTES, reinterpret_cast<cudaStream_t>(stream)>>>(iters, dev_status);
+  if (cudaGetLastError() != cudaSuccess) return HDQT_ERR_CUDA;
+  if (ops_out) *ops_out = 2ll * BM * BN * 32 * (int64_t)iters * sms;
+  return HDQT_OK;
+}

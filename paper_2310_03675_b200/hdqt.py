@@ -29,7 +29,7 @@ EXPORTED = [
     "hdqt_quantize_hadamard", "hdqt_quantize_workspace_bytes", "hdqt_gemm_i8_tiled",
     "hdqt_gemm_i8_workspace_bytes", "hdqt_calibrate_acc_shift", "hdqt_gemm_fwd", "hdqt_gemm_dgrad",
     "hdqt_gemm_wgrad", "hdqt_workspace_bytes", "hdqt_workspace_layout", "hdqt_quantize_hadamard_static",
-    "hdqt_selftest_bounded_wait", "hdqt_conv2d_fwd", "hdqt_conv2d_wgrad",
+    "hdqt_selftest_bounded_wait", "hdqt_conv2d_fwd", "hdqt_conv2d_wgrad", "hdqt_selftest_mma_rate",
 ]
 
 
@@ -93,6 +93,8 @@ def _load() -> C.CDLL:
     lib.hdqt_calibrate_acc_shift.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, sz, vp, vp]
     for name in ("hdqt_gemm_fwd", "hdqt_gemm_dgrad", "hdqt_gemm_wgrad"):
         getattr(lib, name).argtypes = [C.POINTER(GemmDesc), vp, vp, vp, i64, i64, i64, i32, vp, sz, vp, vp]
+    lib.hdqt_selftest_mma_rate.argtypes = [i32, C.POINTER(C.c_int64), vp, vp]
+    lib.hdqt_selftest_mma_rate.restype = C.c_int
     lib.hdqt_selftest_bounded_wait.argtypes = [vp, vp, vp]
     lib.hdqt_selftest_bounded_wait.restype = C.c_int
     for name in ("hdqt_conv2d_fwd", "hdqt_conv2d_wgrad"):
@@ -396,3 +398,18 @@ def conv2d_wgrad(X, G, kernel: int, stride: int = 1, padding: int = 0, desc: Opt
                                  workspace.buf.data_ptr(), workspace.buf.numel(), _ptr(dev_status), _stream()),
            "hdqt_conv2d_wgrad")
     return out, workspace
+
+
+def mma_rate_tops(iters: int = 20000, repeats: int = 3, dev_status=None) -> float:
+    """Integer tensor rate (TOP/s) of back-to-back M128 N256 K32 kind::i8 MMAs on all SMs (no loads, no epilogue),
+    best of `repeats` timed launches: the ceiling of the tiled GEMM at the current clocks."""
+    ops = C.c_int64(0)
+    best = 0.0
+    for _ in range(repeats + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        _check(lib.hdqt_selftest_mma_rate(iters, C.byref(ops), _ptr(dev_status), _stream()), "hdqt_selftest_mma_rate")
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, ops.value / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    return best

@@ -589,3 +589,13 @@ def test_fused_bias_and_relu(hdqt, Nb, D, C, heavy):
     want_b = O.gemm_fwd(X, W, O.fwd_desc(tag_a=0, tag_b=1, bias=bias))
     out_b, _ = hdqt.gemm_fwd(_dev(X), _dev(W), desc=hdqt.default_desc("fwd", bias=bd), dev_status=status)
     assert np.array_equal(out_b.cpu().numpy(), want_b["out"])
+
+
+def test_mma_rate_yardstick_runs_and_is_plausible(hdqt):
+    """The MMA-only loop finishes within its bounded wait and reports a rate of the order of the chip's dense
+    int8 figure (a few POP/s)."""
+    status = hdqt.new_status("cuda")
+    rate = hdqt.mma_rate_tops(iters=4000, repeats=2, dev_status=status)
+    hdqt.check_device_status(status)
+    assert 1000.0 < rate < 6000.0
+    assert hdqt.lib.hdqt_selftest_mma_rate(0, None, None, None) == 1      # invalid argument, nothing launched
