@@ -352,8 +352,10 @@ def gemm_wgrad(X, G, desc: Optional[GemmDesc] = None, w_is_cd: bool = False, wor
 
 # ---- convolution without a materialised patch matrix ------------------------------------------------
 
-def conv2d_out_size(H: int, W: int, kernel: int, stride: int, padding: int):
-    return (H + 2 * padding - kernel) // stride + 1, (W + 2 * padding - kernel) // stride + 1
+def conv2d_out_size(H: int, W: int, kernel, stride: int, padding: int):
+    """Output height and width; `kernel` is an int (square) or a (kh, kw) pair."""
+    kh, kw = (kernel, kernel) if isinstance(kernel, int) else kernel
+    return (H + 2 * padding - kh) // stride + 1, (W + 2 * padding - kw) // stride + 1
 
 
 def conv2d_fwd(X, W, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc] = None, workspace=None,
@@ -365,7 +367,7 @@ def conv2d_fwd(X, W, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc]
     Cout, kh, kw, Cin2 = W.shape
     if Cin2 != Cin:
         raise ValueError("shape mismatch")
-    Ho, Wo = conv2d_out_size(H, Wd, kh, stride, padding)
+    Ho, Wo = conv2d_out_size(H, Wd, (kh, kw), stride, padding)
     g = Conv2dGeom(B, H, Wd, Cin, kh, kw, stride, padding)
     M, N, K = B * Ho * Wo, Cout, kh * kw * Cin
     if workspace is None:
@@ -378,22 +380,24 @@ def conv2d_fwd(X, W, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc]
     return out, workspace
 
 
-def conv2d_wgrad(X, G, kernel: int, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc] = None,
+def conv2d_wgrad(X, G, kernel, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc] = None,
                  workspace=None, dev_status=None, out=None):
-    """dW[Cout,kh,kw,Cin] from X[B,H,W,Cin] and G[B,Ho,Wo,Cout] (both NHWC). Returns (dW, workspace)."""
+    """dW[Cout,kh,kw,Cin] from X[B,H,W,Cin] and G[B,Ho,Wo,Cout] (both NHWC); `kernel` is an int or (kh, kw).
+    Returns (dW, workspace)."""
     _req(X, "X"); _req(G, "G")
     desc = desc or default_desc("wgrad")
     B, H, Wd, Cin = X.shape
     Cout = G.shape[3]
-    Ho, Wo = conv2d_out_size(H, Wd, kernel, stride, padding)
+    kh, kw = (kernel, kernel) if isinstance(kernel, int) else kernel
+    Ho, Wo = conv2d_out_size(H, Wd, (kh, kw), stride, padding)
     if tuple(G.shape[:3]) != (B, Ho, Wo):
         raise ValueError("shape mismatch")
-    g = Conv2dGeom(B, H, Wd, Cin, kernel, kernel, stride, padding)
-    M, N, K = Cout, kernel * kernel * Cin, B * Ho * Wo
+    g = Conv2dGeom(B, H, Wd, Cin, kh, kw, stride, padding)
+    M, N, K = Cout, kh * kw * Cin, B * Ho * Wo
     if workspace is None:
         workspace = Workspace(desc, M, N, K, X.device)
     if out is None:
-        out = torch.empty((Cout, kernel, kernel, Cin), dtype=torch.float32, device=X.device)
+        out = torch.empty((Cout, kh, kw, Cin), dtype=torch.float32, device=X.device)
     _check(lib.hdqt_conv2d_wgrad(C.byref(desc), C.byref(g), X.data_ptr(), G.data_ptr(), out.data_ptr(), Cout,
                                  workspace.buf.data_ptr(), workspace.buf.numel(), _ptr(dev_status), _stream()),
            "hdqt_conv2d_wgrad")

@@ -124,3 +124,51 @@ def test_class_incremental_loop_end_to_end_on_a_small_budget():
                                     batch=32, memory=40, seed=0, test_per_class=4)
     assert res["steps"] == 12 and len(res["accuracy_after_task"]) == 2
     assert all(0.0 <= a <= 1.0 for a in res["accuracy_after_task"])
+
+
+def _patch_matrix_by_loops(x, kh, kw, stride, pad):
+    """Plain-loop patch matrix of an NHWC array (written independently of the harness): row (b, ho, wo), column
+    (i, j, c) with c fastest, zeros outside the image."""
+    B, H, W, C = x.shape
+    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
+    out = np.zeros((B * Ho * Wo, kh * kw * C), dtype=np.float32)
+    for b in range(B):
+        for ho in range(Ho):
+            for wo in range(Wo):
+                r = (b * Ho + ho) * Wo + wo
+                for i in range(kh):
+                    for j in range(kw):
+                        hi, wi = ho * stride + i - pad, wo * stride + j - pad
+                        if 0 <= hi < H and 0 <= wi < W:
+                            out[r, (i * kw + j) * C:(i * kw + j + 1) * C] = x[b, hi, wi]
+    return out, Ho, Wo
+
+
+@pytest.mark.parametrize("B,H,W,C,kh,kw,stride,pad,cout", [(3, 10, 7, 32, 3, 2, 2, 1, 24), (2, 5, 9, 64, 1, 3, 1, 0, 40),
+                                                           (5, 6, 6, 96, 3, 3, 1, 2, 130)])
+def test_implicit_convolution_entry_points_on_odd_geometries(B, H, W, C, kh, kw, stride, pad, cout):
+    """hdqt_conv2d_fwd / hdqt_conv2d_wgrad through the binding on non-square images and kernels, strides, wide
+    padding and ragged row counts, against the oracle on a patch matrix built by plain loops."""
+    from paper_2310_03675_b200 import hdqt
+    rng = np.random.default_rng(B * 100 + H)
+    x = np.maximum(rng.standard_normal((B, H, W, C)), 0).astype(np.float32)
+    w = (rng.standard_normal((cout, kh, kw, C)) * 0.05).astype(np.float32)
+    Xc, Ho, Wo = _patch_matrix_by_loops(x, kh, kw, stride, pad)
+    g = (rng.standard_t(3, size=(B, Ho, Wo, cout)) * 1e-3).astype(np.float32)
+    Wm = w.reshape(cout, -1)
+    status = hdqt.new_status("cuda")
+    xd, wd, gd = (torch.from_numpy(t).cuda() for t in (x, w, g))
+    y, ws = hdqt.conv2d_fwd(xd, wd, stride, pad, desc=hdqt.default_desc("fwd", seed=4), dev_status=status)
+    want = O.gemm_fwd(Xc, Wm.T, O.fwd_desc(seed=4, tag_a=0, tag_b=1))
+    assert np.array_equal(ws.codes_a().cpu().numpy(), want["Aq"])
+    assert np.array_equal(y.cpu().numpy().reshape(-1, cout), want["out"])
+    dw, ws = hdqt.conv2d_wgrad(xd, gd, (kh, kw), stride, pad, desc=hdqt.default_desc("wgrad", seed=4), dev_status=status)
+    hdqt.check_device_status(status)
+    want = O.gemm_wgrad(Xc, g.reshape(-1, cout), O.wgrad_desc(seed=4, tag_a=4, tag_b=5))
+    assert np.array_equal(ws.codes_b().cpu().numpy(), want["Aq"])      # [C, D] layout: operands trade places
+    assert np.array_equal(dw.cpu().numpy().reshape(cout, -1), want["out"].T)
+    # channels not a multiple of 32 are refused on the host
+    bad = torch.zeros((1, 4, 4, 24), device="cuda")
+    with pytest.raises(hdqt.HdqtError) as err:
+        hdqt.conv2d_fwd(bad, torch.zeros((8, 3, 3, 24), device="cuda"), 1, 1)
+    assert err.value.status == 2
