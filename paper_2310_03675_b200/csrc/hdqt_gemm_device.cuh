@@ -495,18 +495,18 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
   }
 }
 
-__device__ __forceinline__ void release_accumulator(const EpiCtx& e, int buf, uint32_t* drains) {
+__device__ __forceinline__ void release_accumulator(const EpiCtx& e, int buf, uint32_t& drain_par) {
   tc_fence_before();
   __syncwarp();
   if (e.lane == 0) mbar_arrive(e.bar_tempty + 8 * buf);
-  ++drains[buf];
+  drain_par ^= 1u << buf;
 }
 
 // Whole block merged (the common case on heavy-tailed operands): no per-tile sums exist, so the registers
 // take the complete accumulator row at once and the accumulator goes back to the MMA issuer before any
 // conversion or store work.
-__device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
-  if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+__device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
+  if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
   tc_fence_after();
   const float scale = dequant_scale(p);
   uint32_t mv[EPI_COLS];
@@ -514,7 +514,7 @@ __device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx
   for (int c = 0; c < EPI_COLS / 16; ++c) HDQT_TMEM_LD16(e.lane_addr + c * 16, (mv + c * 16));
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 16; ++c) HDQT_TMEM_WAIT16((mv + c * 16));
-  release_accumulator(e, 0, drains);
+  release_accumulator(e, 0, drain_par);
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 16; ++c) {
     int val[16];
@@ -565,7 +565,7 @@ __device__ __forceinline__ void packed_accumulate(uint32_t (&S)[EPI_COLS / 2], u
   }
 }
 
-__device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+__device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
   uint32_t S[EPI_COLS / 2];
 #pragma unroll
   for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
@@ -577,44 +577,54 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
   // back to the MMA issuer as soon as the load has landed, before any arithmetic.  (Arithmetic of a warp does
   // not overlap its own TMEM load in flight - measured: it gets slower -, so the load is not split or
   // prefetched; the other epilogue warp of the scheduler fills the load's latency.)
-  for (int ci = 0; ci < job.n_clamp_tiles; ++ci) {
-    const int buf = job.merging ? 1 : (ci & 1);
-    if (!mbar_wait_suspend(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
-    tc_fence_after();
-    if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(2, ci);
-    uint32_t v[EPI_COLS / 2];
-    HDQT_TMEM_LD64_PACK16(e.lane_addr + buf * BN, v);
-    tmem_ld_wait();
-    release_accumulator(e, buf, drains);
-    if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(4, ci);
-    if (e.lane == 0) HDQT_TL(8 + e.grp * 4 + e.q, ci);      // release time of every epilogue warp
-    packed_accumulate(S, v, rng2);
-    if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(5, ci);
-    if (++n_in_S == p.flush_every && ci + 1 < job.n_clamp_tiles) {
-      // widen: park int32 partial sums in the output buffer
-      const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
-      const int64_t gn0 = (int64_t)job.n0 + e.grp * EPI_COLS;
-      const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
-                       (gn0 + EPI_COLS <= p.N);
-      if (gm < p.M) {
+  // widen: park the int32 partial sums in the output buffer (added to what is parked there already)
+  auto park_sums = [&]() {
+    const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
+    const int64_t gn0 = (int64_t)job.n0 + e.grp * EPI_COLS;
+    const bool vec = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
+                     (gn0 + EPI_COLS <= p.N);
+    if (gm < p.M) {
 #pragma unroll
-        for (int i = 0; i < EPI_COLS / 2; i += 2) {
-          int s4[4];
-          s4[0] = (int)(S[i] & 0xFFFFu) - (int)off * n_in_S;
-          s4[1] = (int)(S[i] >> 16) - (int)off * n_in_S;
-          s4[2] = (int)(S[i + 1] & 0xFFFFu) - (int)off * n_in_S;
-          s4[3] = (int)(S[i + 1] >> 16) - (int)off * n_in_S;
-          emit4<false>(p, gm, gn0 + 2 * i, s4, parked, vec, 0.0f);
-        }
+      for (int i = 0; i < EPI_COLS / 2; i += 2) {
+        int s4[4];
+        s4[0] = (int)(S[i] & 0xFFFFu) - (int)off * n_in_S;
+        s4[1] = (int)(S[i] >> 16) - (int)off * n_in_S;
+        s4[2] = (int)(S[i + 1] & 0xFFFFu) - (int)off * n_in_S;
+        s4[3] = (int)(S[i + 1] >> 16) - (int)off * n_in_S;
+        emit4<false>(p, gm, gn0 + 2 * i, s4, parked, vec, 0.0f);
       }
+    }
 #pragma unroll
-      for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+    for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+  };
+  // Two nested loops: the widening step (rare, a lot of code) sits between runs of at most flush_every tiles,
+  // outside the per-tile loop, so that the per-tile loop is one short stretch of code.
+  for (int base = 0; base < job.n_clamp_tiles; base += p.flush_every) {
+    const int run_end = min(job.n_clamp_tiles, base + p.flush_every);
+#pragma unroll 1
+    for (int ci = base; ci < run_end; ++ci) {
+      const int buf = job.merging ? 1 : (ci & 1);
+      if (!mbar_wait_suspend(e.bar_tfull + 8 * buf, (drain_par >> buf) & 1u, e.abort_flag)) return false;
+      tc_fence_after();
+      if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(2, ci);
+      uint32_t v[EPI_COLS / 2];
+      HDQT_TMEM_LD64_PACK16(e.lane_addr + buf * BN, v);
+      tmem_ld_wait();
+      release_accumulator(e, buf, drain_par);
+      if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(4, ci);
+      if (e.lane == 0) HDQT_TL(8 + e.grp * 4 + e.q, ci);      // release time of every epilogue warp
+      packed_accumulate(S, v, rng2);
+      if (e.q == HDQT_TL_Q && e.grp == 0 && e.lane == 0) HDQT_TL(5, ci);
+    }
+    n_in_S = run_end - base;
+    if (run_end < job.n_clamp_tiles) {
+      park_sums();
       n_in_S = 0;
       parked = true;
     }
   }
   if (job.n_merged > 0) {
-    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
     tc_fence_after();
   }
   const float scale = dequant_scale(p);
@@ -625,7 +635,7 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
       HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
       HDQT_TMEM_WAIT16(mv);
       // the last of the merged accumulator is in registers: hand it back to the MMA issuer
-      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drains);
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drain_par);
     }
     int val[16];
 #pragma unroll
@@ -645,21 +655,21 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
 
 // 32-bit path: one register per accumulator element, any b_a and shift r, optional per-tile debug output.
 template <bool kShift, bool kTilesOut>
-__device__ __forceinline__ bool epilogue_wide(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t* drains) {
+__device__ __forceinline__ bool epilogue_wide(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
   int S[EPI_COLS];
 #pragma unroll
   for (int i = 0; i < EPI_COLS; ++i) S[i] = 0;
   const int r = p.acc_shift, lo = p.lo, hi = p.hi;
   for (int ci = 0; ci < job.n_clamp_tiles; ++ci) {
     const int buf = job.merging ? 1 : (ci & 1);
-    if (!mbar_wait(e.bar_tfull + 8 * buf, drains[buf] & 1u, e.abort_flag)) return false;
+    if (!mbar_wait(e.bar_tfull + 8 * buf, (drain_par >> buf) & 1u, e.abort_flag)) return false;
     tc_fence_after();
 #pragma unroll
     for (int c = 0; c < EPI_COLS / 16; ++c) {
       uint32_t v[16];
       HDQT_TMEM_LD16(e.lane_addr + buf * BN + c * 16, v);
       HDQT_TMEM_WAIT16(v);
-      if (c == EPI_COLS / 16 - 1) release_accumulator(e, buf, drains);
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, buf, drain_par);
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const int ct = acc_quant<kShift>((int)v[i], r, lo, hi);
@@ -677,7 +687,7 @@ __device__ __forceinline__ bool epilogue_wide(const GemmParams& p, EpiCtx e, Blo
     }
   }
   if (job.n_merged > 0) {
-    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drains[0] & 1u, e.abort_flag)) return false;
+    if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
     tc_fence_after();
   }
   const float scale = dequant_scale(p);
@@ -690,7 +700,7 @@ __device__ __forceinline__ bool epilogue_wide(const GemmParams& p, EpiCtx e, Blo
       uint32_t mv[16];
       HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
       HDQT_TMEM_WAIT16(mv);
-      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drains);
+      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drain_par);
 #pragma unroll
       for (int i = 0; i < 16; ++i) val[i] += (int)mv[i];
     }

@@ -8,6 +8,7 @@ namespace hdqt {
 
 namespace {
 
+
 // ---- the kernel -----------------------------------------------------------------------------
 // Persistent: one CTA per SM walks over output blocks (block index = blockIdx.x + i*gridDim.x), so that the
 // TMA producer runs ahead into the next block while the epilogue warps drain the previous one, and the
@@ -240,7 +241,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       const uint32_t offset_mma = (uint32_t)p.offset_mma;
       uint32_t s = 0;            // smem stage
       uint32_t full_par = 0;     // parity of the stage's next "full" phase
-      uint32_t fills[2] = {0u, 0u};   // how many times each TMEM accumulator has been handed to the epilogue
+      uint32_t fill_par = 0u;   // bit b: parity of the times TMEM accumulator b has been handed to the epilogue
       uint64_t desc_a = desc_a0, desc_b = desc_b0;
       bool ok = true;
       const int tpa = p.tiles_per_acc;
@@ -285,7 +286,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const int nsub = min(tiles32 - kt0, 4);
             for (int sub = 0; sub < nsub; ++sub) {
               const uint32_t b = (uint32_t)clamp_idx & 1u;
-              if (!mbar_wait_suspend(bar_tempty + 8 * b, (fills[b] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+              if (!mbar_wait_suspend(bar_tempty + 8 * b, ((fill_par >> b) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
               tc_fence_after();
               HDQT_TL(0, clamp_idx);
               const uint32_t d = tmem_base + b * BN;
@@ -293,14 +294,14 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
               tc_mma_i8(d, desc_a + (uint64_t)(2 * sub), desc_b + (uint64_t)(2 * sub), 1u);
               HDQT_TL(1, clamp_idx);
               tc_commit(bar_tfull + 8 * b);
-              ++fills[b];
+              fill_par ^= 1u << b;
               ++clamp_idx;
             }
             if (!ok) break;
           } else if (nib == 0xFu && kt0 + 4 <= tiles32) {
             if (!merged_started) {
               // the merged accumulator (buffer 0) must have been drained by the previous user
-              if (!mbar_wait(bar_tempty, (fills[0] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+              if (!mbar_wait(bar_tempty, (fill_par & 1u) ^ 1u, abort_flag)) { ok = false; break; }
               tc_fence_after();
             }
             tc_mma_i8(tmem_base, desc_a, desc_b, merged_started);
@@ -321,7 +322,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 // merged tiles accumulate in buffer 0; clamp tiles use buffer 1 when merging, else 0 / 1
                 cur_buf = cert ? 0 : (merging ? 1 : (clamp_idx & 1));
                 if (!cert || !merged_started) {
-                  if (!mbar_wait_suspend(bar_tempty + 8 * cur_buf, (fills[cur_buf] & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                  if (!mbar_wait_suspend(bar_tempty + 8 * cur_buf, ((fill_par >> cur_buf) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                   tc_fence_after();
                 }
                 d_tmem = tmem_base + cur_buf * BN;
@@ -348,7 +349,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 if (!cert) {
                   HDQT_TL(1, clamp_idx);
                   tc_commit(bar_tfull + 8 * cur_buf);
-                  ++fills[cur_buf];
+                  fill_par ^= 1u << cur_buf;
                   ++clamp_idx;
                 }
                 j = 0;
@@ -372,7 +373,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (!ok) break;
         if (n_merged > 0) {
           tc_commit(bar_tfull + 0);
-          ++fills[0];
+          fill_par ^= 1u;
         }
         if (p.merge == 1) mbar_arrive(bar_iempty + 8 * slot);
       }
@@ -390,7 +391,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     e.bar_tempty = bar_tempty;
     e.abort_flag = abort_flag;
     e.box = reinterpret_cast<float*>(smem_al + OUT_STAGE_OFF + (warp - NUM_CTRL_WARPS) * OUT_STAGE_WARP);
-    uint32_t drains[2] = {0u, 0u};      // how many times this warp has drained each accumulator
+    uint32_t drain_par = 0u;            // bit b: parity of the times this warp has drained accumulator b
     int ti = 0;
     for (int tile = blockIdx.x; tile < num_items; tile += gridDim.x, ++ti) {
       const ItemRange ir = item_range(tile);
@@ -410,9 +411,9 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       job.m0 = tile_m * BM;
       job.n0 = tile_n * BN;
       bool ok;
-      if (job.n_clamp_tiles == 0 && job.n_merged > 0) ok = epilogue_merged_only(p, e, job, drains);
-      else if (kPacked) ok = epilogue_packed(p, e, job, drains);
-      else ok = epilogue_wide<kShift, kTilesOut>(p, e, job, drains);
+      if (job.n_clamp_tiles == 0 && job.n_merged > 0) ok = epilogue_merged_only(p, e, job, drain_par);
+      else if (kPacked) ok = epilogue_packed(p, e, job, drain_par);
+      else ok = epilogue_wide<kShift, kTilesOut>(p, e, job, drain_par);
       if (!ok) break;
       if (p.merge == 1) {
         __syncwarp();
