@@ -356,7 +356,8 @@ def train_steps_records(torch, dev, steps=20):
     """Training steps per second of the synthetic MLP and CNN workloads and of a class-incremental batch mix
     (new-task samples + replayed exemplars, grown head), every matmul through the library (with measured maxima,
     and with delayed scaling: maxima carried from the previous step, no calibration pass); the fp32 torch step of
-    the same model beside each.  Accuracy needs the long run (`--workload cil`)."""
+    the same model beside each, and every variant once more as a step replayed from CUDA graphs.  Accuracy needs
+    the long run (`--workload cil`)."""
     from paper_2310_03675_b200 import nn as hnn
     out = {}
 
@@ -382,6 +383,11 @@ def train_steps_records(torch, dev, steps=20):
         opt = torch.optim.SGD(model.parameters(), lr=0.01, momentum=0.9)
         ms = time_steps(lambda i: hnn.train_step(model, opt, x, labels, i), 5 * steps)
         rec[name] = {"steps_per_s": 1e3 / ms, "ms_per_step": ms}
+        # the same step replayed from CUDA graphs (random stream advanced by a device-side word)
+        stepper = hnn.GraphedTrainStep(model, opt, x, labels)
+        ms = time_steps(lambda i: stepper(x, labels), 5 * steps)
+        rec[name + "_cuda_graph"] = {"steps_per_s": 1e3 / ms, "ms_per_step": ms}
+        del stepper
     out["mlp_1152_512_256_12_batch256"] = rec
 
     patterns = hnn.class_patterns(100, seed=SEED, device=dev)
@@ -398,6 +404,10 @@ def train_steps_records(torch, dev, steps=20):
         opt = torch.optim.SGD(model.parameters(), lr=0.05, momentum=0.9, weight_decay=2e-4)
         ms = time_steps(lambda i: hnn.cnn_train_step(model, opt, x, labels, i), steps)
         rec[name] = {"steps_per_s": 1e3 / ms, "ms_per_step": ms}
+        stepper = hnn.GraphedTrainStep(model, opt, x, labels)
+        ms = time_steps(lambda i: stepper(x, labels), steps)
+        rec[name + "_cuda_graph"] = {"steps_per_s": 1e3 / ms, "ms_per_step": ms}
+        del stepper
         # class-incremental batch: second task, 64 new samples (classes 20..39) + 64 replayed, head of 40 neurons
         labels_cil = torch.cat([torch.randint(20, 40, (64,), generator=g, device=dev),
                                 torch.randint(0, 20, (64,), generator=g, device=dev)])

@@ -111,6 +111,11 @@ typedef struct hdqt_gemm_desc {
   const uint32_t* amax_hist_in_b;
   uint32_t* amax_hist_out_a;
   uint32_t* amax_hist_out_b;
+  /* Optional device uint32: its value at the time the kernels run is the fourth Philox counter word of both
+     operands' stochastic roundings (0 when NULL).  `seed` is fixed when a call is recorded into a CUDA graph;
+     a caller who replays the graph advances this word on the device instead (one increment per training
+     step), so that no two steps round with the same random numbers.                                          */
+  const uint32_t* philox_offset;
 } hdqt_gemm_desc_t;
 
 #define HDQT_AMAX_HISTORY_WORDS 1024
@@ -152,7 +157,8 @@ hdqt_status_t hdqt_absmax_hadamard(const float* src, int64_t rows, int64_t K,
  *   t = clip*amax, v = (src H) * (2^(bits-1) / t)
  *   nearest   : code = clamp(rint(v))
  *   stochastic: code = clamp(floor((rint(v*2^16) + u16) / 2^16)), u16 = 16 bits of
- *               Philox4x32-10(counter = (g lo, g hi, tag, 0), key = seed), g = idx/8,
+ *               Philox4x32-10(counter = (g lo, g hi, tag, 0), key = seed), g = idx/8 (the GEMM calls put
+ *               the descriptor's philox_offset word in place of the 0),
  *               idx = r*K_pad + k; element idx%8 takes half (idx&1) of word (idx%8)/2
  *   clamp to [-2^(bits-1), 2^(bits-1)-1]; all-zero tensor -> zero codes, step 0.
  *

@@ -128,19 +128,21 @@ def philox4x32_10(c0, c1, c2, c3, k0: int, k1: int):
             c2.astype(np.uint32), c3.astype(np.uint32))
 
 
-def sr_random_u16(seed: int, tag: int, idx: np.ndarray) -> np.ndarray:
+def sr_random_u16(seed: int, tag: int, idx: np.ndarray, stream: int = 0) -> np.ndarray:
     """The 16 random bits that stochastic rounding uses for element `idx`.
 
     idx is the element's linear index in the code layout [rows, K_pad].  Eight
-    consecutive elements share one Philox call: counter = (g_lo, g_hi, tag, 0)
+    consecutive elements share one Philox call: counter = (g_lo, g_hi, tag, stream)
     with g = idx // 8, key = (seed_lo, seed_hi); element e = idx % 8 takes the
-    low (e even) or high (e odd) half of output word e // 2."""
+    low (e even) or high (e odd) half of output word e // 2.  `stream` (32 bits,
+    0 unless the caller advances it, e.g. once per training step) selects one of
+    2^32 independent streams under the same key."""
     idx = np.asarray(idx, dtype=np.uint64)
     g = idx >> np.uint64(3)
     e = (idx & np.uint64(7)).astype(np.int64)
     w = philox4x32_10(g & _MASK32, g >> np.uint64(32),
                       np.full(g.shape, int(tag) & 0xFFFFFFFF, dtype=np.uint64),
-                      np.zeros(g.shape, dtype=np.uint64),
+                      np.full(g.shape, int(stream) & 0xFFFFFFFF, dtype=np.uint64),
                       int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF)
     words = np.stack(w, axis=0).astype(np.uint64)          # [4, ...]
     word = np.take_along_axis(words, (e >> 1)[None, ...], axis=0)[0]
@@ -148,7 +150,7 @@ def sr_random_u16(seed: int, tag: int, idx: np.ndarray) -> np.ndarray:
     return half.astype(np.int64)
 
 
-def sr_random_u16_tensor(seed: int, tag: int, rows: int, K_pad: int) -> np.ndarray:
+def sr_random_u16_tensor(seed: int, tag: int, rows: int, K_pad: int, stream: int = 0) -> np.ndarray:
     """sr_random_u16 for every element of a [rows, K_pad] code tensor, with one
     Philox call per group of eight elements instead of one per element."""
     n = rows * K_pad
@@ -156,7 +158,7 @@ def sr_random_u16_tensor(seed: int, tag: int, rows: int, K_pad: int) -> np.ndarr
     g = np.arange(n // 8, dtype=np.uint64)
     w = philox4x32_10(g & _MASK32, g >> np.uint64(32),
                       np.full(g.shape, int(tag) & 0xFFFFFFFF, dtype=np.uint64),
-                      np.zeros(g.shape, dtype=np.uint64),
+                      np.full(g.shape, int(stream) & 0xFFFFFFFF, dtype=np.uint64),
                       int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF)
     out = np.empty((n // 8, 8), dtype=np.int64)
     for j in range(4):
@@ -170,7 +172,7 @@ def sr_random_u16_tensor(seed: int, tag: int, rows: int, K_pad: int) -> np.ndarr
 # --------------------------------------------------------------------------
 
 def quantize_transformed(xh: np.ndarray, bits: int, clip: float, mode: int,
-                         seed: int = 0, tag: int = 0, amax=None):
+                         seed: int = 0, tag: int = 0, amax=None, stream: int = 0):
     """Quantize an already transformed (and padded) fp32 tensor xh[rows, K_pad].
 
     Returns (codes int8 [rows, K_pad], step fp32, amax fp32).
@@ -208,7 +210,7 @@ def quantize_transformed(xh: np.ndarray, bits: int, clip: float, mode: int,
     elif mode == ROUND_STOCHASTIC:
         v_fx = np.rint((v * F32(65536.0)).astype(F32)).astype(np.int64)
         rows, Kp = xh.shape
-        u16 = sr_random_u16_tensor(seed, tag, rows, Kp)
+        u16 = sr_random_u16_tensor(seed, tag, rows, Kp, stream)
         q = (v_fx + u16) >> 16          # arithmetic shift = floor division
     else:
         raise ValueError("unknown rounding mode")
@@ -218,12 +220,12 @@ def quantize_transformed(xh: np.ndarray, bits: int, clip: float, mode: int,
 
 def quantize_hadamard(src: np.ndarray, had_block: int = 32, bits: int = 4,
                       clip: float = 1.0, mode: int = ROUND_NEAREST,
-                      seed: int = 0, tag: int = 0, amax=None):
+                      seed: int = 0, tag: int = 0, amax=None, stream: int = 0):
     """src[rows, K] (K = contraction dim) -> (codes [rows, K_pad], step, amax).
 
     pad -> block-diagonal FWHT along K -> max calibration -> quantize."""
     xh = fwht_blockdiag(pad_contraction(src, had_block), had_block)
-    return quantize_transformed(xh, bits, clip, mode, seed, tag, amax)
+    return quantize_transformed(xh, bits, clip, mode, seed, tag, amax, stream)
 
 
 # --------------------------------------------------------------------------
@@ -309,13 +311,14 @@ class GemmDesc:
     def __init__(self, in_bits=4, acc_bits=8, acc_tile=32, acc_shift=0,
                  had_block=32, clip_a=1.0, clip_b=1.0,
                  round_a=ROUND_NEAREST, round_b=ROUND_NEAREST,
-                 seed=0, tag_a=0, tag_b=1, bias=None, relu=False):
+                 seed=0, tag_a=0, tag_b=1, bias=None, relu=False, philox_offset=0):
         self.in_bits, self.acc_bits, self.acc_tile = in_bits, acc_bits, acc_tile
         self.acc_shift, self.had_block = acc_shift, had_block
         self.clip_a, self.clip_b = clip_a, clip_b
         self.round_a, self.round_b = round_a, round_b
         self.seed, self.tag_a, self.tag_b = seed, tag_a, tag_b
         self.bias, self.relu = bias, relu
+        self.philox_offset = philox_offset    # fourth Philox counter word of both operands' streams
 
 
 def hdqt_gemm(A_mk: np.ndarray, B_nk: np.ndarray, d: GemmDesc, want_tiles=False):
@@ -323,9 +326,9 @@ def hdqt_gemm(A_mk: np.ndarray, B_nk: np.ndarray, d: GemmDesc, want_tiles=False)
     given with the contraction dimension last.  Returns a dict with every
     intermediate the GPU path is compared on."""
     Aq, sa, amax_a = quantize_hadamard(A_mk, d.had_block, d.in_bits, d.clip_a,
-                                       d.round_a, d.seed, d.tag_a)
+                                       d.round_a, d.seed, d.tag_a, stream=d.philox_offset)
     Bq, sb, amax_b = quantize_hadamard(B_nk, d.had_block, d.in_bits, d.clip_b,
-                                       d.round_b, d.seed, d.tag_b)
+                                       d.round_b, d.seed, d.tag_b, stream=d.philox_offset)
     out, S, tiles = gemm_i8_tiled(Aq, Bq, sa, sb, d.acc_bits, d.acc_tile,
                                   d.acc_shift, d.had_block, want_tiles, d.bias, d.relu)
     return dict(out=out, S=S, tiles=tiles, Aq=Aq, Bq=Bq, step_a=sa, step_b=sb,

@@ -112,7 +112,7 @@ extern "C" hdqt_status_t hdqt_quantize_hadamard(const float* src, int64_t rows, 
   a.amax_in = amax_in;
   a.amax_slot = reinterpret_cast<float*>(workspace);
   a.codes = codes; a.step_out = step_out; a.tile_norms = tile_norms;
-  return launch_calibrate_quantize(&a, 1, had_block, bits, seed,
+  return launch_calibrate_quantize(&a, 1, had_block, bits, seed, nullptr,
                                    reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(workspace) + 256),
                                    dev_status, reinterpret_cast<cudaStream_t>(stream));
 }
@@ -218,7 +218,7 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
   ops[1] = QuantOperand{gB.src, gB.rows, K, gB.ld_row, gB.ld_k, gB.conv, clipB, roundB, tagB, amaxB, histInB, histOutB,
                         reinterpret_cast<float*>(ws + L.amax_b), reinterpret_cast<int8_t*>(ws + L.codes_b),
                         reinterpret_cast<float*>(ws + L.step_b), normsB};
-  st = launch_calibrate_quantize(ops, 2, d->had_block, d->in_bits, d->seed,
+  st = launch_calibrate_quantize(ops, 2, d->had_block, d->in_bits, d->seed, d->philox_offset,
                                  reinterpret_cast<uint32_t*>(ws + L.gemm_ws), dev_status, s);
   if (st != HDQT_OK) return st;
   return gemm_i8_tiled_impl(reinterpret_cast<int8_t*>(ws + L.codes_a), reinterpret_cast<int8_t*>(ws + L.codes_b),

@@ -149,7 +149,8 @@ hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t l
 // share had_block, bits and seed: at most one launch per pass and memory layout.
 // partials: scratch of n_ops * kMaxPartials uint32.
 hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int32_t had_block, int32_t bits,
-                                        uint64_t seed, uint32_t* partials, int32_t* dev_status, cudaStream_t s);
+                                        uint64_t seed, const uint32_t* philox_offset, uint32_t* partials,
+                                        int32_t* dev_status, cudaStream_t s);
 
 // hdqt_gemm_i8_tiled plus an optional output-column bias (fp32 [N]); HDQT_FLAG_RELU in `flags` clamps at zero
 hdqt_status_t gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const float* step_a, const float* step_b,

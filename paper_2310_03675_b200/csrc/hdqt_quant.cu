@@ -200,6 +200,7 @@ struct QuantParams {
   bool sr_magic;     // |v| < 64 guaranteed: fixed-point conversion through the fp32 adder
   bool zero_all;     // degenerate scale (all-zero or non-finite tensor): every code is 0
   uint32_t tag;
+  uint32_t stream;          // fourth Philox counter word (0, or the caller's device-side stream offset)
   const PhiloxKeys* keys;   // the launch's round keys (a kernel parameter)
 };
 
@@ -225,7 +226,7 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams
       t[i] = __vimin_s32_relu(q, p.rng);
     }
   } else {
-    const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, 0u, *p.keys);
+    const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, p.stream, *p.keys);
     // s = rint(v * 2^16) + u16 + (offset << 16), a Q.16 fixed-point integer; code + offset = floor(s / 2^16), clamped
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -270,7 +271,7 @@ __device__ __forceinline__ void dispatch_mode(const QuantParams& p, int had_bloc
 }
 
 __device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bits, float clip, int mode,
-                                                   const PhiloxKeys* keys, uint32_t tag) {
+                                                   const PhiloxKeys* keys, uint32_t tag, uint32_t stream) {
   QuantParams p;
   const int off = 1 << (bits - 1);
   p.m = qs.m;
@@ -283,6 +284,7 @@ __device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bit
   p.sr_magic = ((float)off <= 32.0f * clip);  // |v| <= 32 (1 + eps)
   p.zero_all = qs.zero || qs.bad;
   p.keys = keys;
+  p.stream = stream;
   p.tag = tag;
   return p;
 }
@@ -321,6 +323,7 @@ struct QuantBatch {
   int32_t n_ops;
   int32_t had_block;
   int32_t bits;
+  const uint32_t* stream;   // optional device word: fourth Philox counter word of the stochastic roundings
 };
 
 // which operand this thread block works on, and its block index within that operand
@@ -474,7 +477,7 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   int local_block;
   const QuantOp& op = my_operand(b, local_block);
   const QuantScale qs = resolve_scale(op, local_block, b.bits, dev_status);
-  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag);
+  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag, b.stream ? __ldg(b.stream) : 0u);
   const float* __restrict__ src = op.src;
   int8_t* __restrict__ codes = op.codes;
   const int64_t K = op.K, ld_row = op.ld;
@@ -538,7 +541,7 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
   int local_block;
   const QuantOp& op = my_operand(b, local_block);
   const QuantScale qs = resolve_scale(op, local_block, b.bits, dev_status);
-  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag);
+  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag, b.stream ? __ldg(b.stream) : 0u);
   const float* __restrict__ src = op.src;
   int8_t* __restrict__ codes = op.codes;
   const int64_t K = op.K, K_pad = op.K_pad, ld_row = op.ld, rows = op.rows;
@@ -712,7 +715,7 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
   int local_block;
   const QuantOp& op = my_operand(b, local_block);
   const QuantScale qs = resolve_scale(op, local_block, b.bits, dev_status);
-  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag);
+  const QuantParams p = make_params(qs, b.bits, op.clip, op.mode, &keys, op.tag, b.stream ? __ldg(b.stream) : 0u);
   const float* __restrict__ src = op.src;
   int8_t* __restrict__ codes = op.codes;
   int32_t* __restrict__ tile_norms = op.tile_norms;
@@ -878,7 +881,8 @@ hdqt_status_t launch_absmax(const float* src, int64_t rows, int64_t K, int64_t l
 }
 
 hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int32_t had_block, int32_t bits,
-                                        uint64_t seed, uint32_t* partials, int32_t* dev_status, cudaStream_t s) {
+                                        uint64_t seed, const uint32_t* philox_offset, uint32_t* partials,
+                                        int32_t* dev_status, cudaStream_t s) {
   if (n_ops < 1 || n_ops > kMaxOps) return HDQT_ERR_INVALID_ARG;
   QuantOp op[kMaxOps];
   for (int i = 0; i < n_ops; ++i) {
@@ -920,6 +924,7 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
     QuantBatch b{};
     b.had_block = had_block;
     b.bits = bits;
+    b.stream = philox_offset;
     int grid = 0;
     for (int i = 0; i < n_ops; ++i) {
       const int v = (ops[i].ld_k != 1) ? 2 : (ops[i].tile_norms != nullptr ? 1 : 0);
@@ -1011,6 +1016,6 @@ extern "C" hdqt_status_t hdqt_quantize_hadamard_static(const float* src, int64_t
   a.amax_in = nullptr;
   a.amax_slot = reinterpret_cast<float*>(scratch);
   a.codes = codes; a.step_out = step_out; a.tile_norms = tile_norms;
-  return hdqt::launch_calibrate_quantize(&a, 1, had_block, bits, seed, reinterpret_cast<uint32_t*>(scratch + 256),
+  return hdqt::launch_calibrate_quantize(&a, 1, had_block, bits, seed, nullptr, reinterpret_cast<uint32_t*>(scratch + 256),
                                          dev_status, reinterpret_cast<cudaStream_t>(stream));
 }

@@ -43,6 +43,7 @@ class GemmDesc(C.Structure):
         ("flags", C.c_uint32), ("bias", C.c_void_p),
         ("amax_hist_in_a", C.c_void_p), ("amax_hist_in_b", C.c_void_p),
         ("amax_hist_out_a", C.c_void_p), ("amax_hist_out_b", C.c_void_p),
+        ("philox_offset", C.c_void_p),
     ]
 
 
@@ -146,7 +147,8 @@ def default_desc(kind: str, **overrides) -> GemmDesc:
     d = GemmDesc()
     lib.hdqt_default_desc(C.byref(d), {"fwd": 0, "dgrad": 1, "wgrad": 2}[kind])
     for k, v in overrides.items():
-        if k in ("amax_a", "amax_b", "bias", "amax_hist_in_a", "amax_hist_in_b", "amax_hist_out_a", "amax_hist_out_b"):
+        if k in ("amax_a", "amax_b", "bias", "amax_hist_in_a", "amax_hist_in_b", "amax_hist_out_a", "amax_hist_out_b",
+                 "philox_offset"):
             v = _ptr(v)
         setattr(d, k, v)
     return d
@@ -378,6 +380,20 @@ def conv2d_fwd(X, W, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc]
                                workspace.buf.data_ptr(), workspace.buf.numel(), _ptr(dev_status), _stream()),
            "hdqt_conv2d_fwd")
     return out, workspace
+
+
+def conv2d_dgrad(G, W, padding: int = 0, desc: Optional[GemmDesc] = None, workspace=None, dev_status=None, out=None):
+    """dX[B,H,W,Cin] of a stride-1 convolution from G[B,Ho,Wo,Cout] (NHWC, Cout % 32 == 0) and W[Cout,kh,kw,Cin]:
+    the input gradient is itself a convolution, of G with the kernel rotated by 180 degrees and padding
+    k-1-padding, so it runs through hdqt_conv2d_fwd with the dgrad roles (stochastic rounding on G, nearest on
+    W): contraction over (kh, kw, cout), no patch-matrix gradient and no scatter-add.  Returns (dX, workspace)."""
+    _req(G, "G"); _req(W, "W")
+    desc = desc or default_desc("dgrad")
+    Cout, kh, kw, Cin = W.shape
+    if G.shape[3] != Cout or kh - 1 - padding != kw - 1 - padding or kh - 1 - padding < 0:
+        raise ValueError("shape mismatch")
+    w_rot = W.flip(1, 2).permute(3, 1, 2, 0).contiguous()          # [Cin, kh, kw, Cout]
+    return conv2d_fwd(G, w_rot, 1, kh - 1 - padding, desc=desc, workspace=workspace, dev_status=dev_status, out=out)
 
 
 def conv2d_wgrad(X, G, kernel, stride: int = 1, padding: int = 0, desc: Optional[GemmDesc] = None,

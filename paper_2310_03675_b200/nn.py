@@ -163,6 +163,65 @@ def train_step(model: Mlp, opt: torch.optim.Optimizer, x, labels, step: int):
     return loss
 
 
+class GraphedTrainStep:
+    """One training step (forward, loss, backward, optimiser step) of a fixed-shape model recorded into CUDA
+    graphs and replayed: the library calls never synchronise the host and allocate nothing per call, so a whole
+    step is one graph launch instead of several hundred kernel launches with their host-side cost.
+
+    The Philox seed of a recorded call is fixed, so the stochastic roundings of successive replays are told apart
+    on the device: every quantized layer gets `philox_offset` = a device counter that the graph itself increments
+    once per step (step k rounds with (seed, offset) = (base_step, k)).  Two graphs are recorded and replayed
+    alternately, because delayed scaling ping-pongs between two history buffers per tensor.
+
+    `forward(x)` maps the static input batch to logits; `warmup` eager steps run first (they are real training
+    steps: optimiser state and workspaces must exist before the recording)."""
+
+    def __init__(self, model: torch.nn.Module, opt: torch.optim.Optimizer, x: torch.Tensor, labels: torch.Tensor,
+                 forward=None, base_step: int = 0, warmup: int = 3):
+        self.model, self.opt = model, opt
+        self.forward = forward if forward is not None else model
+        dev = x.device
+        self.counter = torch.zeros(1, dtype=torch.int32, device=dev)
+        for m in model.modules():
+            if isinstance(m, (HdqtLinear, HdqtConv2d)):
+                m.over = dict(m.over, philox_offset=self.counter)
+                m.step = base_step
+        self.x, self.labels = x.clone(), labels.clone()
+        self.steps = 0
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.stream(side):
+            for _ in range(warmup):
+                self._body()
+        torch.cuda.current_stream(dev).wait_stream(side)
+        self.graphs, self.losses = [], []
+        for _ in range(2):
+            g = torch.cuda.CUDAGraph()
+            opt.zero_grad(set_to_none=True)
+            with torch.cuda.graph(g, pool=self.graphs[0].pool() if self.graphs else None):
+                loss = self._body()
+            self.graphs.append(g)
+            self.losses.append(loss)
+        self.steps = warmup
+
+    def _body(self):
+        self.opt.zero_grad(set_to_none=True)
+        loss = torch.nn.functional.cross_entropy(self.forward(self.x), self.labels)
+        loss.backward()
+        self.opt.step()
+        self.counter += 1
+        return loss
+
+    def __call__(self, x: torch.Tensor, labels: torch.Tensor) -> torch.Tensor:
+        """Copies the batch into the static buffers and replays one step; returns the (static) loss tensor."""
+        self.x.copy_(x, non_blocking=True)
+        self.labels.copy_(labels, non_blocking=True)
+        i = self.steps & 1
+        self.graphs[i].replay()
+        self.steps += 1
+        return self.losses[i]
+
+
 # ---- convolution as an im2col GEMM -------------------------------------------------------------------
 # The transform and the quantizer act along the contraction dimension of the matmul a convolution lowers to
 # (paper Section 3: Z = X W for every layer): rows = output positions (batch x Ho x Wo), contraction =
@@ -221,8 +280,9 @@ class HdqtConv2dFunction(torch.autograd.Function):
     """y = conv2d(x, w) (no bias) with the forward, dX and dW products as HDQT GEMMs on the patch (im2col)
     matrix.  With cin % 32 == 0 the forward and dW products gather the patches straight from the NHWC
     activation inside the library's transform/quantize kernels (no patch matrix is materialised); other layers
-    (the 3-channel stem) build the matrix with torch copies.  dX is the dgrad GEMM followed by the scatter-add
-    of the patch-matrix gradient."""
+    (the 3-channel stem) build the matrix with torch copies.  dX of a stride-1 layer (cout % 32 == 0) is the
+    convolution of G with the rotated kernel through the same implicit path (contraction over kh x kw x cout);
+    strided and 1x1 layers take the dgrad GEMM on the patch matrix followed by its scatter-add."""
 
     @staticmethod
     def forward(ctx, x, w, stride: int, padding: int, layer_id: int, seed: int, over: dict, implicit: bool):
@@ -259,9 +319,15 @@ class HdqtConv2dFunction(torch.autograd.Function):
         dx = dw = None
         if ctx.needs_input_grad[0]:
             d = _desc("dgrad", layer_id, seed, g.device, **over)
-            dxc, _ = hdqt.gemm_dgrad(g2d, wm, desc=d, w_is_cd=True,
-                                     workspace=_workspace(d, g2d.shape[0], wm.shape[1], Cout, g.device))
-            dx = _col2im(dxc, xshape, kh, stride, padding, Ho, Wo)
+            if implicit and stride == 1 and kh > 1 and Cout % 32 == 0:
+                # the input gradient of a stride-1 convolution is a convolution of G with the rotated kernel
+                dxn, _ = hdqt.conv2d_dgrad(gn, wm.view(Cout, kh, kw, Cin), padding, desc=d,
+                                           workspace=_workspace(d, B * xshape[2] * xshape[3], Cin, kh * kw * Cout, g.device))
+                dx = dxn.permute(0, 3, 1, 2)
+            else:
+                dxc, _ = hdqt.gemm_dgrad(g2d, wm, desc=d, w_is_cd=True,
+                                         workspace=_workspace(d, g2d.shape[0], wm.shape[1], Cout, g.device))
+                dx = _col2im(dxc, xshape, kh, stride, padding, Ho, Wo)
         if ctx.needs_input_grad[1]:
             d = _desc("wgrad", layer_id, seed, g.device, **over)
             if implicit:

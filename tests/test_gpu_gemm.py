@@ -599,3 +599,41 @@ def test_mma_rate_yardstick_runs_and_is_plausible(hdqt):
     hdqt.check_device_status(status)
     assert 1000.0 < rate < 6000.0
     assert hdqt.lib.hdqt_selftest_mma_rate(0, None, None, None) == 1      # invalid argument, nothing launched
+
+
+@pytest.mark.parametrize("kind,shape", [("dgrad", (70, 96, 200)), ("wgrad", (64, 300, 40)), ("wgrad", (2048, 160, 4100))])
+def test_device_side_philox_offset(hdqt, kind, shape):
+    """The descriptor's device word is the fourth Philox counter word of every stochastic rounding of the call:
+    both operand layouts (and the tile-norm variant of the large weight-gradient case) agree with the oracle's
+    `philox_offset`, the word is read when the kernels run (not when the call is made), and offset 0 is the
+    plain stream."""
+    Nb, D, Cc = shape
+    X, W, G = inputs.activations(Nb, D, seed=1), inputs.weights(D, Cc, seed=2), inputs.gradients(Nb, Cc, seed=3)
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    status = hdqt.new_status("cuda")
+    codes = {}
+    for off in (0, 7, 0x80000001):
+        word.fill_(off - (1 << 32) if off >= (1 << 31) else off)
+        d = hdqt.default_desc(kind, seed=5, philox_offset=word)
+        if kind == "dgrad":
+            out, ws = hdqt.gemm_dgrad(_dev(G), _dev(W), desc=d, dev_status=status)
+            want = O.gemm_dgrad(G, W, O.dgrad_desc(seed=5, tag_a=2, tag_b=3, philox_offset=off))
+        else:
+            out, ws = hdqt.gemm_wgrad(_dev(X), _dev(G), desc=d, dev_status=status)
+            want = O.gemm_wgrad(X, G, O.wgrad_desc(seed=5, tag_a=4, tag_b=5, philox_offset=off))
+        hdqt.check_device_status(status)
+        assert np.array_equal(ws.codes_a().cpu().numpy(), want["Aq"])
+        assert np.array_equal(ws.codes_b().cpu().numpy(), want["Bq"])
+        assert np.array_equal(out.cpu().numpy(), want["out"])
+        codes[off] = ws.codes_a().cpu().numpy().copy()
+    assert not np.array_equal(codes[0], codes[7])
+    # stream-ordered: the word is changed after the call was enqueued behind a change, not at call time
+    word.fill_(7)
+    d = hdqt.default_desc(kind, seed=5, philox_offset=word)
+    if kind == "dgrad":
+        _, ws = hdqt.gemm_dgrad(_dev(G), _dev(W), desc=d, dev_status=status)
+    else:
+        _, ws = hdqt.gemm_wgrad(_dev(X), _dev(G), desc=d, dev_status=status)
+    got = ws.codes_a().clone()
+    word.fill_(0)
+    assert np.array_equal(got.cpu().numpy(), codes[7])

@@ -82,3 +82,61 @@ def test_delayed_scaling_in_the_linear_layer_matches_the_oracle_with_carried_max
     first = O.gemm_fwd(X0, W, O.fwd_desc(seed=0, tag_a=base, tag_b=base + 1))["out"]
     assert np.array_equal(outs[0][0], first)
     hnn.reset_delayed_scaling()
+
+
+def test_graphed_step_equals_eager_steps():
+    """A training step replayed from a CUDA graph, with the random stream advanced by the device-side Philox word,
+    gives the same losses bit for bit as eager steps that pass the same (seed, offset) pairs."""
+    from paper_2310_03675_b200 import nn as hnn
+    dev = torch.device("cuda")
+    sizes = (96, 64, 12)
+
+    def make():
+        torch.manual_seed(0)
+        m = hnn.Mlp(sizes).to(dev)
+        return m, torch.optim.SGD(m.parameters(), lr=0.05, momentum=0.9)
+
+    batches = [hnn.sensor_window_batch(64, sizes[0], sizes[-1], seed=i, device=dev) for i in range(9)]
+    # eager: every layer reads the step from a device word that the loop advances
+    m1, o1 = make()
+    word = torch.zeros(1, dtype=torch.int32, device=dev)
+    for l in m1.layers:
+        l.over = dict(l.over, philox_offset=word)
+    eager = []
+    for x, y in batches:
+        eager.append(float(hnn.train_step(m1, o1, x, y, step=0).detach()))
+        word += 1
+    # graphed: three eager warm-up steps inside the constructor, then replays
+    m2, o2 = make()
+    stepper = None
+    graphed = []
+    for i, (x, y) in enumerate(batches):
+        if i < 3:
+            continue
+        if stepper is None:
+            # the constructor's warm-up steps train on its example batch: feed it the first three batches in turn
+            stepper = _warm_graphed(hnn, m2, o2, batches[:3])
+            graphed = list(stepper.warm_losses)
+        graphed.append(float(stepper(x, y).detach()))
+    assert graphed == eager
+    assert len(set(eager)) == len(eager)
+
+
+def _warm_graphed(hnn, model, opt, first):
+    """GraphedTrainStep whose warm-up steps run on the given batches (one each)."""
+    it = iter(first)
+    losses = []
+
+    class Stepper(hnn.GraphedTrainStep):
+        def _body(self):
+            if len(losses) < len(first):
+                x, y = next(it)
+                self.x.copy_(x); self.labels.copy_(y)
+            loss = super()._body()
+            if len(losses) < len(first):
+                losses.append(float(loss.detach()))
+            return loss
+
+    s = Stepper(model, opt, first[0][0], first[0][1], warmup=len(first))
+    s.warm_losses = losses
+    return s

@@ -458,3 +458,25 @@ def test_bias_and_relu_tail_is_plain_fp32_arithmetic():
     a = O.gemm_fwd(X, W, O.fwd_desc())["out"]
     b = O.gemm_fwd(X, W, O.fwd_desc(bias=bias, relu=True))["out"]
     assert np.array_equal(b, np.maximum((a + bias).astype(np.float32), 0))
+
+
+def test_sr_stream_word_is_the_fourth_philox_counter_word():
+    """`stream` selects the fourth counter word of the Philox call behind the 16 rounding bits: stream 0 is the
+    plain generator, any other value gives different bits for the same (seed, tag, index), and the choice reaches
+    the codes of a stochastic quantization but not those of a nearest one."""
+    idx = np.arange(64, dtype=np.uint64) + 8 * 12345
+    base = O.sr_random_u16(3, 9, idx)
+    assert np.array_equal(base, O.sr_random_u16(3, 9, idx, stream=0))
+    other = O.sr_random_u16(3, 9, idx, stream=2)
+    assert (base != other).mean() > 0.9
+    g = int(idx[8] >> 3)
+    w = O.philox4x32_10(np.array([g], np.uint32), np.array([0], np.uint32), np.array([9], np.uint32),
+                        np.array([2], np.uint32), 3, 0)
+    assert other[8] == int(w[0][0]) & 0xFFFF and other[11] == int(w[1][0]) >> 16
+    assert np.array_equal(O.sr_random_u16_tensor(3, 9, 4, 32, stream=2).ravel()[:64], O.sr_random_u16(3, 9, np.arange(64), stream=2))
+    x = np.random.default_rng(0).standard_normal((8, 64)).astype(np.float32)
+    q0 = O.quantize_hadamard(x, mode=O.ROUND_STOCHASTIC, seed=1, tag=2)[0]
+    q1 = O.quantize_hadamard(x, mode=O.ROUND_STOCHASTIC, seed=1, tag=2, stream=1)[0]
+    assert not np.array_equal(q0, q1) and np.abs(q0.astype(int) - q1.astype(int)).max() <= 1
+    n0 = O.quantize_hadamard(x, mode=O.ROUND_NEAREST, seed=1, tag=2)[0]
+    assert np.array_equal(n0, O.quantize_hadamard(x, mode=O.ROUND_NEAREST, seed=1, tag=2, stream=1)[0])
