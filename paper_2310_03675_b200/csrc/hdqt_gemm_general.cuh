@@ -277,7 +277,27 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           uint32_t nib = 0;
           if (p.merge == 2) nib = 0xFu;
           else if (nibble_ok) nib = (cert_mask[kb >> 3] >> ((kb & 7) * 4)) & 0xFu;
-          if (!merging && tpa == 1 && offset_mma) {
+          if (!merging && tpa == 1 && offset_mma && kt0 + 4 <= tiles32 && (clamp_idx & 1) == 0) {
+            // A whole stage of clamp-path tiles, straight-line: this thread's instructions are the pace of the
+            // ring (each costs it tens of clocks beside the epilogue warps of its scheduler), so accumulator,
+            // K slice and barrier parity of the four tiles are compile-time constants.  Each accumulator is
+            // handed over twice per stage, which leaves the hand-over parities as they were.
+            const uint32_t p0 = (fill_par & 1u) ^ 1u, p1 = ((fill_par >> 1) & 1u) ^ 1u;
+#pragma unroll
+            for (int sub = 0; sub < 4; ++sub) {
+              const uint32_t b = (uint32_t)sub & 1u;
+              const uint32_t par = (b ? p1 : p0) ^ (uint32_t)(sub >> 1);
+              if (!mbar_wait_suspend(bar_tempty + 8 * b, par, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              HDQT_TL(0, clamp_idx + sub);
+              tc_mma_i8_new(tmem_base + b * BN, desc_offs_a, desc_offs_b);
+              tc_mma_i8_acc(tmem_base + b * BN, desc_a + (uint64_t)(2 * sub), desc_b + (uint64_t)(2 * sub));
+              HDQT_TL(1, clamp_idx + sub);
+              tc_commit(bar_tfull + 8 * b);
+            }
+            if (!ok) break;
+            clamp_idx += 4;
+          } else if (!merging && tpa == 1 && offset_mma) {
             // Every tile of this block takes the clamp path of the 16-bit-lane epilogue: a short, branch-free
             // sequence per tile.  (This thread shares its scheduler with two epilogue warps; every instruction
             // it spends between two tiles is taken from them, and they are the slowest of the eight.  Issuing
