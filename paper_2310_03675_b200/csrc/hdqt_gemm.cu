@@ -174,10 +174,10 @@ bool make_operand_map(CUtensorMap* map, const int8_t* base, int64_t rows, int64_
   return r == CUDA_SUCCESS;
 }
 
-template <bool kPacked, bool kShift, bool kTilesOut>
+template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false>
 hdqt_status_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, dim3 grid,
                              cudaStream_t s) {
-  auto kern = gemm_i8_tiled_kernel<kPacked, kShift, kTilesOut>;
+  auto kern = gemm_i8_tiled_kernel<kPacked, kShift, kTilesOut, kDeep>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return cuda_failure(e, "cudaFuncSetAttribute(gemm)");
   kern<<<grid, GEMM_THREADS, SMEM_BYTES, s>>>(ma, mb, p);
@@ -384,7 +384,12 @@ hdqt_status_t hdqt::gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const
                      : launch_variant<false, false, true>(ma, mb, p, grid, s);
   }
   hdqt_status_t st;
-  if (packed) st = launch_variant<true, false, false>(ma, mb, p, grid, s);
+  // more clamp-path tiles per work item than the 16-bit lanes hold: the variant with a second set of lanes (up
+  // to 256 x flush_every tiles; beyond that the plain variant parks partial sums in the output buffer)
+  const int64_t tiles_per_item = p.split_k > 1 ? (int64_t)p.split_kblocks * 4 / tpa : num_acc;
+  const bool deep = packed && tiles_per_item > p.flush_every && tiles_per_item <= 256 * (int64_t)p.flush_every;
+  if (packed && deep) st = launch_variant<true, false, false, true>(ma, mb, p, grid, s);
+  else if (packed) st = launch_variant<true, false, false>(ma, mb, p, grid, s);
   else st = acc_shift ? launch_variant<false, true, false>(ma, mb, p, grid, s)
                       : launch_variant<false, false, false>(ma, mb, p, grid, s);
   if (st == HDQT_OK && p.split_k > 1) {

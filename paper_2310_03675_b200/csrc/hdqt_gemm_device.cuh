@@ -432,6 +432,7 @@ struct EpiCtx {               // constants of one epilogue warp
   volatile int* abort_flag;
   float* box;                 // this warp's 32 x 16 fp32 staging box in shared memory
   int q, grp, lane;
+  float scale;                // dequantisation scale of the launch (formed once per warp, not per output block)
 };
 
 struct BlockJob {             // one output block as seen by the epilogue
@@ -456,6 +457,7 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
                                             int (&val)[16], bool parked, float scale, bool raw = false) {
   const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
   const int64_t gn = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16;
+  if (gn >= p.N) return;      // (warp-uniform) columns beyond the matrix: nothing to write
   if (job.atomic) {
     // split-K: integer partial sums of this K range (the buffer was cleared before the launch)
     if (gm < p.M) {
@@ -534,7 +536,7 @@ __device__ __forceinline__ void release_accumulator(const EpiCtx& e, int buf, ui
 __device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
   if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
   tc_fence_after();
-  const float scale = dequant_scale(p);
+  const float scale = e.scale;
   uint32_t mv[EPI_COLS];
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 16; ++c) HDQT_TMEM_LD16(e.lane_addr + c * 16, (mv + c * 16));
@@ -591,10 +593,18 @@ __device__ __forceinline__ void packed_accumulate(uint32_t (&S)[EPI_COLS / 2], u
   }
 }
 
+// kDeep (contractions of more than flush_every tiles, chosen by the host): a second set of 16-bit lanes takes the
+// high bytes of the lane sums every flush_every tiles (sum = low + 256 * high), so that nothing is parked in memory
+// for up to 256 * flush_every tiles; it costs 64 more registers, which is why it is a variant of its own.
+template <bool kDeep>
 __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
   uint32_t S[EPI_COLS / 2];
+  uint32_t Shi[kDeep ? EPI_COLS / 2 : 1];
 #pragma unroll
   for (int i = 0; i < EPI_COLS / 2; ++i) S[i] = 0u;
+#pragma unroll
+  for (int i = 0; i < (kDeep ? EPI_COLS / 2 : 1); ++i) Shi[i] = 0u;
+  int n_deep = 0;        // tiles whose high bytes have moved to Shi
   const uint32_t off = (uint32_t)(-p.lo);                    // c + off lies in [0, hi - lo]
   const uint32_t rng2 = (uint32_t)(p.hi - p.lo) | ((uint32_t)(p.hi - p.lo) << 16);
   int n_in_S = 0;
@@ -659,16 +669,26 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
     }
     n_in_S = run_end - base;
     if (run_end < job.n_clamp_tiles) {
-      park_sums();
-      n_in_S = 0;
-      parked = true;
+      if constexpr (kDeep) {
+#pragma unroll
+        for (int i = 0; i < EPI_COLS / 2; ++i) {
+          Shi[i] += (S[i] >> 8) & 0x00FF00FFu;
+          S[i] &= 0x00FF00FFu;
+        }
+        n_deep += n_in_S;
+      } else {
+        park_sums();
+        n_in_S = 0;
+        parked = true;
+      }
     }
   }
+  if constexpr (kDeep) n_in_S += n_deep;     // every tile's offset is still in the two lane sets
   if (job.n_merged > 0) {
     if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
     tc_fence_after();
   }
-  const float scale = dequant_scale(p);
+  const float scale = e.scale;
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 16; ++c) {
     uint32_t mv[16];
@@ -684,6 +704,11 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
       const uint32_t sp = S[c * 8 + i];
       val[2 * i] = (int)(sp & 0xFFFFu) - (int)off * n_in_S;
       val[2 * i + 1] = (int)(sp >> 16) - (int)off * n_in_S;
+      if constexpr (kDeep) {
+        const uint32_t hp = Shi[c * 8 + i];
+        val[2 * i] += (int)((hp & 0xFFFFu) << 8);
+        val[2 * i + 1] += (int)((hp >> 16) << 8);
+      }
       if (job.n_merged > 0) {
         val[2 * i] += (int)mv[2 * i];
         val[2 * i + 1] += (int)mv[2 * i + 1];
@@ -731,7 +756,7 @@ __device__ __forceinline__ bool epilogue_wide(const GemmParams& p, EpiCtx e, Blo
     if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
     tc_fence_after();
   }
-  const float scale = dequant_scale(p);
+  const float scale = e.scale;
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 16; ++c) {
     int val[16];

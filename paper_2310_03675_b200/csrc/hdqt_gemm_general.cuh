@@ -21,6 +21,7 @@ namespace {
 //
 // kPacked: the per-tile sums fit 16 bits and b_a <= 8, r = 0: TMEM is read with two columns packed
 //          per register, clamp and add work on 16-bit lane pairs (half the ALU work per element).
+// kDeep:   with kPacked, for contractions longer than flush_every tiles: two-level lane sums (see epilogue_packed).
 // otherwise: one 32-bit register per accumulator element, any b_a and r.
 
 struct TileInfo {                       // what the certificate warp publishes per output block
@@ -55,7 +56,7 @@ __device__ __forceinline__ void block_coords(const GemmParams& p, int i, int til
   }
 }
 
-template <bool kPacked, bool kShift, bool kTilesOut>
+template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
@@ -411,6 +412,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     e.bar_tempty = bar_tempty;
     e.abort_flag = abort_flag;
     e.box = reinterpret_cast<float*>(smem_al + OUT_STAGE_OFF + (warp - NUM_CTRL_WARPS) * OUT_STAGE_WARP);
+    e.scale = dequant_scale(p);
     uint32_t drain_par = 0u;            // bit b: parity of the times this warp has drained accumulator b
     int ti = 0;
     for (int tile = blockIdx.x; tile < num_items; tile += gridDim.x, ++ti) {
@@ -432,7 +434,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       job.n0 = tile_n * BN;
       bool ok;
       if (job.n_clamp_tiles == 0 && job.n_merged > 0) ok = epilogue_merged_only(p, e, job, drain_par);
-      else if (kPacked) ok = epilogue_packed(p, e, job, drain_par);
+      else if (kPacked) ok = epilogue_packed<kDeep>(p, e, job, drain_par);
       else ok = epilogue_wide<kShift, kTilesOut>(p, e, job, drain_par);
       if (!ok) break;
       if (p.merge == 1) {

@@ -304,6 +304,7 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     e.abort_flag = abort_flag;
     e.box = reinterpret_cast<float*>(smem_raw + P_OUT_OFF + (warp - 2) * OUT_STAGE_WARP);
     const float scale = dequant_scale(p);
+    e.scale = scale;
     int bi = 0;
     for (int i = pair_id; i < num_blocks; i += num_pairs, ++bi) {
       const int buf = bi & 1;

@@ -637,3 +637,33 @@ def test_device_side_philox_offset(hdqt, kind, shape):
     got = ws.codes_a().clone()
     word.fill_(0)
     assert np.array_equal(got.cpu().numpy(), codes[7])
+
+
+@pytest.mark.parametrize("K,acc_bits", [(32 * 260, 8), (32 * 700, 8), (32 * 1100, 5)])
+def test_long_contraction_keeps_lane_sums_in_registers(hdqt, K, acc_bits):
+    """More clamp-path tiles per output block than the 16-bit lane sums hold (256 at b_a = 8): the variant with
+    a second set of lanes (low byte / high bytes) must give the same integers as the oracle, for operands that
+    never clamp, that clamp often (sums of a lane run close to the lane limit) and for all-saturated tiles,
+    with split-K switched off so that a work item really spans the whole contraction."""
+    rng = np.random.default_rng(K)
+    M, N = 200, 300
+    one = torch.ones(1, device="cuda")
+    flags = hdqt.FLAG_NO_MERGE | hdqt.FLAG_NO_SPLIT_K
+    status = hdqt.new_status("cuda")
+    for kind in ("calm", "wild", "saturated"):
+        if kind == "calm":
+            Aq = np.clip(np.rint(rng.standard_normal((M, K)) * 1.2), -8, 7).astype(np.int8)
+            Bq = np.clip(np.rint(rng.standard_normal((N, K)) * 1.2), -8, 7).astype(np.int8)
+        elif kind == "wild":
+            Aq, Bq = _codes(rng, M, K), _codes(rng, N, K)
+        else:
+            Aq, Bq = np.full((M, K), 7, np.int8), np.full((N, K), 7, np.int8)     # every tile sum clamps to the top
+            Bq[::2] = -8                                                          # ... or to the bottom
+        want_out, want_S, _ = O.gemm_i8_tiled(Aq, Bq, 1.0, 1.0, acc_bits)
+        out, S, _ = hdqt.gemm_i8_tiled(_dev(Aq), _dev(Bq), one, one, acc_bits, want_S=True, flags=flags,
+                                       dev_status=status)
+        hdqt.check_device_status(status)
+        assert np.array_equal(S.cpu().numpy().astype(np.int64), want_S), kind
+        assert np.array_equal(out.cpu().numpy(), want_out), kind
+    if acc_bits == 8:
+        assert int(np.abs(want_S).max()) == 128 * (K // 32)       # the saturated case reaches the largest sum there is
