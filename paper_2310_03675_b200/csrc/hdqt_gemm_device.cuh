@@ -453,6 +453,10 @@ __device__ __forceinline__ float dequant_scale(const GemmParams& p) {
 // store instruction writes 8 rows x 64 contiguous bytes (whole sectors) instead of 32 rows x 16 bytes;
 // stores are fire-and-forget, so the box can be reused as soon as the warp has read it back.
 // raw = true parks the integer sums themselves (as bit patterns) for a later fix-up pass instead.
+// kDirect: every thread stores its own row with 16-byte vector stores instead (no staging box, no warp syncs:
+// less code and fewer registers around a long main loop; less efficient stores, so only where the final pass is
+// rare: the long-contraction variant).
+template <bool kDirect = false>
 __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e, const BlockJob& job, int c,
                                             int (&val)[16], bool parked, float scale, bool raw = false) {
   const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
@@ -470,6 +474,17 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
   }
   const bool staged = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
                       (gn + 16 <= p.N);    // warp-uniform
+  if (kDirect && staged) {
+    if (gm < p.M) {
+#pragma unroll
+      for (int i = 0; i < 16; i += 4) {
+        int s4[4] = {val[i], val[i + 1], val[i + 2], val[i + 3]};
+        if (raw) emit4<false>(p, gm, gn + i, s4, parked, true, scale);
+        else emit4<true>(p, gm, gn + i, s4, parked, true, scale);
+      }
+    }
+    return;
+  }
   if (staged) {
     if (gm < p.M && (parked || (p.S_out != nullptr && !raw))) {
 #pragma unroll
@@ -533,6 +548,7 @@ __device__ __forceinline__ void release_accumulator(const EpiCtx& e, int buf, ui
 // Whole block merged (the common case on heavy-tailed operands): no per-tile sums exist, so the registers
 // take the complete accumulator row at once and the accumulator goes back to the MMA issuer before any
 // conversion or store work.
+template <bool kDirect = false>
 __device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
   if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
   tc_fence_after();
@@ -548,7 +564,7 @@ __device__ __forceinline__ bool epilogue_merged_only(const GemmParams& p, EpiCtx
     int val[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) val[i] = (int)mv[c * 16 + i];
-    store_chunk(p, e, job, c, val, false, scale);
+    store_chunk<kDirect>(p, e, job, c, val, false, scale);
   }
   return true;
 }
@@ -596,7 +612,7 @@ __device__ __forceinline__ void packed_accumulate(uint32_t (&S)[EPI_COLS / 2], u
 // kDeep (contractions of more than flush_every tiles, chosen by the host): a second set of 16-bit lanes takes the
 // high bytes of the lane sums every flush_every tiles (sum = low + 256 * high), so that nothing is parked in memory
 // for up to 256 * flush_every tiles; it costs 64 more registers, which is why it is a variant of its own.
-template <bool kDeep>
+template <bool kDeep, bool kMerge = true>
 __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
   uint32_t S[EPI_COLS / 2];
   uint32_t Shi[kDeep ? EPI_COLS / 2 : 1];
@@ -653,7 +669,7 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
       return true;
     };
     int ci = base;
-    if (!job.merging && (base & 1) == 0) {
+    if (!(kMerge && job.merging) && (base & 1) == 0) {
       // tiles alternate between the two accumulators: pairs with the accumulator index fixed at compile time
       // (barrier and TMEM addresses then stay in uniform registers: 740 -> 876 TOPS at 8192^3; four per
       // iteration gave nothing more)
@@ -665,7 +681,7 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
     }
 #pragma unroll 1
     for (; ci < run_end; ++ci) {
-      if (!one_tile(ci, job.merging ? 1 : (ci & 1))) return false;
+      if (!one_tile(ci, (kMerge && job.merging) ? 1 : (ci & 1))) return false;
     }
     n_in_S = run_end - base;
     if (run_end < job.n_clamp_tiles) {
@@ -684,7 +700,7 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
     }
   }
   if constexpr (kDeep) n_in_S += n_deep;     // every tile's offset is still in the two lane sets
-  if (job.n_merged > 0) {
+  if (kMerge && job.n_merged > 0) {
     if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
     tc_fence_after();
   }
@@ -692,7 +708,7 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 16; ++c) {
     uint32_t mv[16];
-    if (job.n_merged > 0) {   // uniform
+    if (kMerge && job.n_merged > 0) {   // uniform
       HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
       HDQT_TMEM_WAIT16(mv);
       // the last of the merged accumulator is in registers: hand it back to the MMA issuer
@@ -709,12 +725,12 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
         val[2 * i] += (int)((hp & 0xFFFFu) << 8);
         val[2 * i + 1] += (int)((hp >> 16) << 8);
       }
-      if (job.n_merged > 0) {
+      if (kMerge && job.n_merged > 0) {
         val[2 * i] += (int)mv[2 * i];
         val[2 * i + 1] += (int)mv[2 * i + 1];
       }
     }
-    store_chunk(p, e, job, c, val, parked, scale);
+    store_chunk<kDeep>(p, e, job, c, val, parked, scale);
   }
   return true;
 }

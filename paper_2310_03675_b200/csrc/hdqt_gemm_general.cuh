@@ -22,6 +22,7 @@ namespace {
 // kPacked: the per-tile sums fit 16 bits and b_a <= 8, r = 0: TMEM is read with two columns packed
 //          per register, clamp and add work on 16-bit lane pairs (half the ALU work per element).
 // kDeep:   with kPacked, for contractions longer than flush_every tiles: two-level lane sums (see epilogue_packed).
+// kMerge:  false = the launch merges no tiles; the merged paths are compiled out.
 // otherwise: one 32-bit register per accumulator element, any b_a and r.
 
 struct TileInfo {                       // what the certificate warp publishes per output block
@@ -56,7 +57,7 @@ __device__ __forceinline__ void block_coords(const GemmParams& p, int i, int til
   }
 }
 
-template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false>
+template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false, bool kMerge = true>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
@@ -79,6 +80,10 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   TileInfo* tile_info = reinterpret_cast<TileInfo*>(smem_al + STAGES * STAGE_BYTES + 256);   // [2]
 
+  // kMerge = false (launches in which no tile is merged): all code of the merged paths drops out.  The per-tile
+  // loops of the clamp path are sensitive to the size of the code around them (removing the unused staging-box
+  // store of the merged-only epilogue from the long-contraction variant alone was worth 13 %).
+  const int merge_mode = kMerge ? p.merge : 0;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int tiles_m = (int)((p.M + BM - 1) / BM), tiles_n = (int)((p.N + BN - 1) / BN);
@@ -145,8 +150,8 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   // A block merges its certified tiles only when few tiles need the clamp path (that path is
   // single-buffered while merging).
   auto block_merges = [&](int n_uncert) {
-    return (p.merge == 2) ||
-           (p.merge == 1 && (int64_t)n_uncert * 256 <= (int64_t)p.merge_max_uncert_256 * num_acc);
+    return (merge_mode == 2) ||
+           (merge_mode == 1 && (int64_t)n_uncert * 256 <= (int64_t)p.merge_max_uncert_256 * num_acc);
   };
 
   if (warp < NUM_CTRL_WARPS) {
@@ -184,7 +189,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     // bit a is set iff every 32-wide sub-tile of accumulator tile a satisfies
     // max_row ||a||^2 * max_col ||b||^2 <= (hi / tiles_per_acc)^2, so |P| <= hi for the whole block
     // (Cauchy-Schwarz) and the clamp is the identity there.
-    if (p.merge == 1) {
+    if (merge_mode == 1) {
       int ti = 0;
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++ti) {
         const int slot = ti & 1;
@@ -253,19 +258,19 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const int tiles32 = ir.t_end;      // end of this item's K range, in 32-wide tiles
         const int num_acc = ir.n_acc;      // (shadows the block-wide count: accumulator tiles of this item)
         const int slot = ti & 1;
-        int n_uncert = (p.merge == 2) ? 0 : num_acc;
-        if (p.merge == 1) {
+        int n_uncert = (merge_mode == 2) ? 0 : num_acc;
+        if (merge_mode == 1) {
           if (!mbar_wait(bar_ifull + 8 * slot, ((uint32_t)ti >> 1) & 1u, abort_flag)) { ok = false; break; }
           n_uncert = *reinterpret_cast<volatile int32_t*>(&tile_info[slot].n_uncert);
         }
         const bool merging = block_merges(n_uncert);
         const int n_merged = merging ? num_acc - n_uncert : 0;
         const uint32_t* cert_mask = tile_info[slot].mask;
-        const bool nibble_ok = (p.merge == 2) || (merging && p.merge == 1 && tpa == 1);
+        const bool nibble_ok = (merge_mode == 2) || (merging && merge_mode == 1 && tpa == 1);
         int j = 0;                 // position inside the current accumulator tile
         int acc = 0;               // accumulator tile index
         int clamp_idx = 0;         // index among this block's tiles that take the clamp path
-        bool cert = (p.merge == 2);
+        bool cert = (merge_mode == 2);
         uint32_t merged_started = 0;
         uint32_t d_tmem = tmem_base;
         int cur_buf = 0;
@@ -276,7 +281,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           const uint32_t par_next = (s + 1 == STAGES) ? (full_par ^ 1u) : full_par;
           const int kt0 = kb * 4;
           uint32_t nib = 0;
-          if (p.merge == 2) nib = 0xFu;
+          if (merge_mode == 2) nib = 0xFu;
           else if (nibble_ok) nib = (cert_mask[kb >> 3] >> ((kb & 7) * 4)) & 0xFu;
           if (!merging && tpa == 1 && offset_mma && kt0 + 4 <= tiles32 && (clamp_idx & 1) == 0) {
             // A whole stage of clamp-path tiles, straight-line: this thread's instructions are the pace of the
@@ -335,7 +340,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const int kt1 = min(tiles32, kt0 + 4);
             for (int kt = kt0; kt < kt1; ++kt) {
               if (j == 0) {
-                if (p.merge == 2) {
+                if (merge_mode == 2) {
                   cert = true;
                 } else if (merging) {
                   cert = (cert_mask[acc >> 5] >> (acc & 31)) & 1u;
@@ -396,7 +401,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           tc_commit(bar_tfull + 0);
           fill_par ^= 1u;
         }
-        if (p.merge == 1) mbar_arrive(bar_iempty + 8 * slot);
+        if (merge_mode == 1) mbar_arrive(bar_iempty + 8 * slot);
       }
     }
   }
@@ -418,8 +423,8 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     for (int tile = blockIdx.x; tile < num_items; tile += gridDim.x, ++ti) {
       const ItemRange ir = item_range(tile);
       const int slot = ti & 1;
-      int n_uncert = (p.merge == 2) ? 0 : ir.n_acc;
-      if (p.merge == 1) {
+      int n_uncert = (merge_mode == 2) ? 0 : ir.n_acc;
+      if (merge_mode == 1) {
         if (!mbar_wait_yield<128>(bar_ifull + 8 * slot, ((uint32_t)ti >> 1) & 1u, abort_flag)) break;
         n_uncert = *reinterpret_cast<volatile int32_t*>(&tile_info[slot].n_uncert);
       }
@@ -433,11 +438,11 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       job.m0 = tile_m * BM;
       job.n0 = tile_n * BN;
       bool ok;
-      if (job.n_clamp_tiles == 0 && job.n_merged > 0) ok = epilogue_merged_only(p, e, job, drain_par);
-      else if (kPacked) ok = epilogue_packed<kDeep>(p, e, job, drain_par);
+      if (kMerge && job.n_clamp_tiles == 0 && job.n_merged > 0) ok = epilogue_merged_only<kDeep>(p, e, job, drain_par);
+      else if (kPacked) ok = epilogue_packed<kDeep, kMerge>(p, e, job, drain_par);
       else ok = epilogue_wide<kShift, kTilesOut>(p, e, job, drain_par);
       if (!ok) break;
-      if (p.merge == 1) {
+      if (merge_mode == 1) {
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_iempty + 8 * slot);
       }
