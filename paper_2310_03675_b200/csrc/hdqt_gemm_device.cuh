@@ -529,6 +529,82 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
   }
 }
 
+// The common case of the staged store with everything that does not depend on the column chunk formed once per
+// output block: addresses of this lane's box slots and output rows, row predicates, the fp32 tail's flags.  A
+// chunk is then ~70 instructions without a branch (the general store_chunk: ~200 with 27 branches, and the final
+// pass of a block was bound by instruction fetch).  Usable for chunks that lie inside the matrix when the output
+// is 16-byte aligned and nothing is parked, raw, atomic or wanted as integers.
+struct FastStore {
+  float* out0;                 // output address of this lane's first row group, first chunk
+  int64_t row_step;            // 8 rows further
+  uint32_t sts[4];             // shared-memory addresses of the four 16-byte slots this lane writes
+  uint32_t lds[4];             // ... and of the four it reads back (one per row group)
+  const float* bias0;          // bias of this lane's four columns in chunk 0, or null
+  bool row_ok[4];
+  bool relu;
+  bool usable;
+  int chunks_inside;           // chunks [0, chunks_inside) lie wholly inside the matrix
+  bool ragged;                 // ... and one more lies partly inside
+};
+
+__device__ __forceinline__ FastStore make_fast_store(const GemmParams& p, const EpiCtx& e, const BlockJob& job,
+                                                     bool parked) {
+  FastStore f;
+  const int64_t gn0 = (int64_t)job.n0 + e.grp * EPI_COLS;
+  f.usable = !parked && !job.atomic && p.S_out == nullptr && ((p.ld_out & 3) == 0) &&
+             ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) && ((reinterpret_cast<uintptr_t>(p.bias) & 15) == 0);
+  const int64_t left = p.N - gn0;
+  f.chunks_inside = left <= 0 ? 0 : (left >= EPI_COLS ? EPI_COLS / 16 : (int)(left >> 4));
+  f.ragged = left > 0 && left < EPI_COLS && (left & 15) != 0;
+  const int sub = e.lane >> 2, quad = e.lane & 3;
+  const int64_t row0 = (int64_t)job.m0 + e.q * 32 + sub;
+  f.out0 = p.out + row0 * p.ld_out + gn0 + quad * 4;
+  f.row_step = 8 * p.ld_out;
+  const uint32_t box = smem_u32(e.box);
+  const int rot = (e.lane >> 1) & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f.sts[i] = box + (uint32_t)(e.lane * 64 + (((i + rot) & 3) << 4));
+    const int rloc = 8 * i + sub;
+    f.lds[i] = box + (uint32_t)(rloc * 64 + (((quad + ((rloc >> 1) & 3)) & 3) << 4));
+    f.row_ok[i] = row0 + 8 * i < p.M;
+  }
+  f.bias0 = p.bias != nullptr ? p.bias + gn0 + quad * 4 : nullptr;
+  f.relu = p.relu != 0;
+  return f;
+}
+
+__device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+
+// integer sums of columns [16c, 16c+16) of this thread's row -> fp32 output, chunk c inside the matrix
+__device__ __forceinline__ void store_chunk_fast(const FastStore& f, int c, const int (&val)[16], float scale) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    sts128(f.sts[i], __fmul_rn((float)val[4 * i], scale), __fmul_rn((float)val[4 * i + 1], scale),
+           __fmul_rn((float)val[4 * i + 2], scale), __fmul_rn((float)val[4 * i + 3], scale));
+  }
+  __syncwarp();
+  float4 b4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+  if (f.bias0 != nullptr) b4 = __ldg(reinterpret_cast<const float4*>(f.bias0 + c * 16));
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float4 v = lds128(f.lds[i]);
+    if (f.bias0 != nullptr) {
+      v.x = __fadd_rn(v.x, b4.x); v.y = __fadd_rn(v.y, b4.y); v.z = __fadd_rn(v.z, b4.z); v.w = __fadd_rn(v.w, b4.w);
+    }
+    if (f.relu) { v.x = fmaxf(v.x, 0.0f); v.y = fmaxf(v.y, 0.0f); v.z = fmaxf(v.z, 0.0f); v.w = fmaxf(v.w, 0.0f); }
+    if (f.row_ok[i]) *reinterpret_cast<float4*>(f.out0 + i * f.row_step + c * 16) = v;
+  }
+  __syncwarp();
+}
+
 // one elected lane arrives once the whole warp is here (elect.sync converges the warp; no divergent branch)
 __device__ __forceinline__ void warp_arrive_one(uint32_t bar) {
   asm volatile(
@@ -704,34 +780,45 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
     if (!mbar_wait_yield<64>(e.bar_tfull + 0, drain_par & 1u, e.abort_flag)) return false;
     tc_fence_after();
   }
+  const FastStore fast = make_fast_store(p, e, job, parked);
   const float scale = e.scale;
+  // the chunks of one output block, with the store routine chosen once for all of them (two separate stretches
+  // of code: the common one stays compact)
+  auto final_pass = [&]<bool kFast>() {
 #pragma unroll
-  for (int c = 0; c < EPI_COLS / 16; ++c) {
-    uint32_t mv[16];
-    if (kMerge && job.n_merged > 0) {   // uniform
-      HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
-      HDQT_TMEM_WAIT16(mv);
-      // the last of the merged accumulator is in registers: hand it back to the MMA issuer
-      if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drain_par);
-    }
-    int val[16];
+    for (int c = 0; c < EPI_COLS / 16; ++c) {
+      uint32_t mv[16];
+      if (kMerge && job.n_merged > 0) {   // uniform
+        HDQT_TMEM_LD16(e.lane_addr + c * 16, mv);
+        HDQT_TMEM_WAIT16(mv);
+        // the last of the merged accumulator is in registers: hand it back to the MMA issuer
+        if (c == EPI_COLS / 16 - 1) release_accumulator(e, 0, drain_par);
+      }
+      int val[16];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const uint32_t sp = S[c * 8 + i];
-      val[2 * i] = (int)(sp & 0xFFFFu) - (int)off * n_in_S;
-      val[2 * i + 1] = (int)(sp >> 16) - (int)off * n_in_S;
-      if constexpr (kDeep) {
-        const uint32_t hp = Shi[c * 8 + i];
-        val[2 * i] += (int)((hp & 0xFFFFu) << 8);
-        val[2 * i + 1] += (int)((hp >> 16) << 8);
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t sp = S[c * 8 + i];
+        val[2 * i] = (int)(sp & 0xFFFFu) - (int)off * n_in_S;
+        val[2 * i + 1] = (int)(sp >> 16) - (int)off * n_in_S;
+        if constexpr (kDeep) {
+          const uint32_t hp = Shi[c * 8 + i];
+          val[2 * i] += (int)((hp & 0xFFFFu) << 8);
+          val[2 * i + 1] += (int)((hp >> 16) << 8);
+        }
+        if (kMerge && job.n_merged > 0) {
+          val[2 * i] += (int)mv[2 * i];
+          val[2 * i + 1] += (int)mv[2 * i + 1];
+        }
       }
-      if (kMerge && job.n_merged > 0) {
-        val[2 * i] += (int)mv[2 * i];
-        val[2 * i + 1] += (int)mv[2 * i + 1];
+      if constexpr (kFast) {
+        if (c < fast.chunks_inside) store_chunk_fast(fast, c, val, scale);   // (the rest lies beyond the matrix)
+      } else {
+        store_chunk<kDeep>(p, e, job, c, val, parked, scale);
       }
     }
-    store_chunk<kDeep>(p, e, job, c, val, parked, scale);
-  }
+  };
+  if (!kDeep && fast.usable && !fast.ragged) final_pass.template operator()<true>();
+  else final_pass.template operator()<false>();
   return true;
 }
 
