@@ -238,7 +238,8 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   if (warp == 0) {
     // ------------------------------ TMA producer (both CTAs) ------------------
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0;           // stages issued so far (for the drain after a timeout)
+      uint32_t ps = 0, pe_par = 1u;   // stage slot and the parity its "empty" barrier is waited on with
       bool ok = true;
       for (int i = pair_id; i < num_blocks && ok; i += num_pairs) {
         int tm, tn;
@@ -246,12 +247,12 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         const int a_row0 = tm * PAIR_M + (int)cta_rank * BM;
         const int b_row0 = tn * BN + (int)cta_rank * (BN / 2);
         for (int kb = 0; kb < num_kblocks; ++kb, ++it) {
-          const uint32_t s = it % P_STAGES;
-          if (!mbar_wait(bar_empty + 8 * s, ((it / P_STAGES) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          if (leader) mbar_expect_tx(bar_full + 8 * s, 2 * P_STAGE_BYTES);   // collects both CTAs' bytes
-          const uint32_t dst = smem_base + s * P_STAGE_BYTES;
-          tma_load_2d_pair(dst, &map_a, kb * BKB, a_row0, bar_full + 8 * s);
-          tma_load_2d_pair(dst + A_STAGE, &map_b, kb * BKB, b_row0, bar_full + 8 * s);
+          if (!mbar_try_wait(bar_empty + 8 * ps, pe_par) && !mbar_wait(bar_empty + 8 * ps, pe_par, abort_flag)) { ok = false; break; }
+          if (leader) mbar_expect_tx(bar_full + 8 * ps, 2 * P_STAGE_BYTES);   // collects both CTAs' bytes
+          const uint32_t dst = smem_base + ps * P_STAGE_BYTES;
+          tma_load_2d_pair(dst, &map_a, kb * BKB, a_row0, bar_full + 8 * ps);
+          tma_load_2d_pair(dst + A_STAGE, &map_b, kb * BKB, b_row0, bar_full + 8 * ps);
+          if (++ps == P_STAGES) { ps = 0; pe_par ^= 1u; }
         }
       }
       if (*abort_flag && leader) {
@@ -264,30 +265,67 @@ gemm_i8_merged_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   } else if (warp == 1) {
     // ------------------------------ MMA issuer (leader only) ------------------
     if (lane == 0 && leader) {
-      uint32_t it = 0;
+      // The tensor pipe takes one MMA while it works on another, so whatever this thread does between the last MMA
+      // of a stage and the first of the next must fit into one MMA's time: stage index, barrier addresses, parity and
+      // descriptors advance incrementally (no division by the stage count, no descriptor rebuilt), and whole stages
+      // take no test on the tile count.
+      const uint64_t da0 = make_smem_desc(smem_base), db0 = make_smem_desc(smem_base + A_STAGE);
+      uint64_t da = da0, db = db0;
+      uint32_t s = 0, full_par = 0u;
+      uint32_t fb = bar_full, eb = bar_empty;
+      const int full_stages = p.tiles32 >> 2;
       int bi = 0;
       bool ok = true;
+      auto next_stage = [&]() {
+        if (++s == P_STAGES) {
+          s = 0; full_par ^= 1u; da = da0; db = db0; fb = bar_full; eb = bar_empty;
+        } else {
+          da += (uint64_t)(P_STAGE_BYTES >> 4); db += (uint64_t)(P_STAGE_BYTES >> 4); fb += 8; eb += 8;
+        }
+      };
       for (int i = pair_id; i < num_blocks && ok; i += num_pairs, ++bi) {
         const int buf = bi & 1;
         if (!mbar_wait(bar_tempty + 8 * buf, (((uint32_t)bi >> 1) & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
-        for (int kb = 0; kb < num_kblocks; ++kb, ++it) {
-          const uint32_t s = it % P_STAGES;
-          if (!mbar_wait(bar_full + 8 * s, (it / P_STAGES) & 1u, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const uint64_t da = make_smem_desc(smem_base + s * P_STAGE_BYTES);
-          const uint64_t db = make_smem_desc(smem_base + s * P_STAGE_BYTES + A_STAGE);
-          if (kb * 4 + 4 <= p.tiles32) {
-            tc_mma_i8_pair(d_tmem, da, db, kb > 0 ? 1u : 0u);
-            tc_mma_i8_pair(d_tmem, da + 2, db + 2, 1u);
-            tc_mma_i8_pair(d_tmem, da + 4, db + 4, 1u);
-            tc_mma_i8_pair(d_tmem, da + 6, db + 6, 1u);
-          } else {
-            for (int sub = 0; kb * 4 + sub < p.tiles32; ++sub)
-              tc_mma_i8_pair(d_tmem, da + 2 * sub, db + 2 * sub, (kb > 0 || sub > 0) ? 1u : 0u);
+        uint32_t acc = 0u;
+        for (int kb = 0; kb < full_stages; ++kb) {
+          if (s == 0 && kb + P_STAGES <= full_stages) {
+            // one turn of the stage ring with every address a compile-time offset
+#pragma unroll
+            for (int j = 0; j < P_STAGES; ++j) {
+              if (!mbar_try_wait(bar_full + 8 * j, full_par) && !mbar_wait(bar_full + 8 * j, full_par, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              const uint64_t o = (uint64_t)(j * (P_STAGE_BYTES >> 4));
+              tc_mma_i8_pair(d_tmem, da0 + o, db0 + o, acc);
+              tc_mma_i8_pair(d_tmem, da0 + o + 2, db0 + o + 2, 1u);
+              tc_mma_i8_pair(d_tmem, da0 + o + 4, db0 + o + 4, 1u);
+              tc_mma_i8_pair(d_tmem, da0 + o + 6, db0 + o + 6, 1u);
+              acc = 1u;
+              tc_commit_pair(bar_empty + 8 * j);
+            }
+            if (!ok) break;
+            full_par ^= 1u;
+            kb += P_STAGES - 1;
+            continue;
           }
-          tc_commit_pair(bar_empty + 8 * s);
+          if (!mbar_try_wait(fb, full_par) && !mbar_wait(fb, full_par, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          tc_mma_i8_pair(d_tmem, da, db, acc);
+          tc_mma_i8_pair(d_tmem, da + 2, db + 2, 1u);
+          tc_mma_i8_pair(d_tmem, da + 4, db + 4, 1u);
+          tc_mma_i8_pair(d_tmem, da + 6, db + 6, 1u);
+          acc = 1u;
+          tc_commit_pair(eb);
+          next_stage();
+        }
+        if (ok && full_stages < num_kblocks) {       // ragged last stage
+          if (!mbar_wait(fb, full_par, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          for (int sub = 0; full_stages * 4 + sub < p.tiles32; ++sub)
+            tc_mma_i8_pair(d_tmem, da + 2 * sub, db + 2 * sub, (acc != 0u || sub > 0) ? 1u : 0u);
+          tc_commit_pair(eb);
+          next_stage();
         }
         if (ok) tc_commit_pair(bar_tfull + 8 * buf);
       }
