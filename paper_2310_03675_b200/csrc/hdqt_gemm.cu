@@ -339,10 +339,10 @@ hdqt_status_t hdqt::gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const
       return HDQT_ERR_CUDA;
   }
 
-  // Large problems (at least 8 output blocks per SM; below that the extra launches cost more than they gain)
+  // Large problems (at least 2 output blocks per SM; below that the extra launches cost more than they gain)
   // with clamp-free tiles: the cta_group::2 kernel takes the blocks whose K tiles are all, or all but a few,
   // certified (a fix-up pass repairs the few), the general kernel takes the rest.
-  const bool split = (p.merge != 0) && !tiles_out && num_blocks >= 8 * (int64_t)sms && sms >= 2 && workspace != nullptr;
+  const bool split = (p.merge != 0) && !tiles_out && num_blocks >= 2 * (int64_t)sms && sms >= 2 && workspace != nullptr;
   if (split) {
     const SplitLayout L = split_layout(M, N);
     if (L.npb > INT32_MAX / 4) return HDQT_ERR_UNSUPPORTED;
