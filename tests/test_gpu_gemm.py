@@ -566,7 +566,7 @@ def test_bounded_waits_run_out_and_report_timeout(hdqt):
 
 
 @pytest.mark.parametrize("Nb,D,C,heavy", [(64, 96, 40, False), (300, 561, 130, False), (128 * 37 + 50, 1024, 256 * 33 + 24, True),
-                                          (70, 32 * 300, 50, False)])
+                                          (70, 32 * 300, 50, False), (200, 160, 144, False), (700, 4608, 512, False)])
 def test_fused_bias_and_relu(hdqt, Nb, D, C, heavy):
     """Forward product with the bias and ReLU folded into the dequantising epilogue: small blocks, the work split of
     large problems (pair kernel, fix-up pass, general kernel) and split-K all apply the same fp32 tail."""
