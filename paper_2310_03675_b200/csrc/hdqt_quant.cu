@@ -213,7 +213,10 @@ __device__ __forceinline__ uint32_t pack4_offset(const int (&t)[8], int base, ui
 // codes of 8 consecutive elements as two packed words; `g` = (linear index of the first element) / 8.
 // kMode: 0 = nearest, 1 = stochastic with the fixed-point conversion through the fp32 adder (|v| < 64
 // guaranteed), 2 = stochastic with a float-to-int conversion (any v; a quarter of the arithmetic rate).
-template <int kMode>
+// kPerm (stochastic modes): clamp the fixed-point sum itself and gather byte 2 of four sums with byte permutes
+// instead of shifting every sum down (one instruction per element less; used by the K-contiguous kernels - in the
+// K-strided kernel, which runs at its register limit, it made the nearest body 13 % slower).
+template <int kMode, bool kPerm = false>
 __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams& p, uint64_t g, uint32_t& w0,
                                           uint32_t& w1) {
   int t[8];
@@ -228,6 +231,7 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams
   } else {
     const Philox4 rnd = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.tag, p.stream, *p.keys);
     // s = rint(v * 2^16) + u16 + (offset << 16), a Q.16 fixed-point integer; code + offset = floor(s / 2^16), clamped
+    const int rng16 = (p.rng << 16) | 0xFFFF;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float v = __fmul_rn(x[i], p.m);
@@ -240,34 +244,44 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], const QuantParams
       } else {
         s = __float2int_rn(__fmul_rn(v, 65536.0f)) + u16 + p.off16;
       }
-      t[i] = __vimin_s32_relu(s >> 16, p.rng);
+      // kPerm: s clamped to [0, rng * 2^16 + 0xFFFF], its byte 2 is code + offset
+      t[i] = kPerm ? __vimin_s32_relu(s, rng16) : __vimin_s32_relu(s >> 16, p.rng);
     }
   }
-  w0 = pack4_offset(t, 0, p.addc);
-  w1 = pack4_offset(t, 4, p.addc);
+  if (kMode != 0 && kPerm) {
+    const uint32_t a01 = __byte_perm((uint32_t)t[0], (uint32_t)t[1], 0x0062), a23 = __byte_perm((uint32_t)t[2], (uint32_t)t[3], 0x0062);
+    const uint32_t a45 = __byte_perm((uint32_t)t[4], (uint32_t)t[5], 0x0062), a67 = __byte_perm((uint32_t)t[6], (uint32_t)t[7], 0x0062);
+    w0 = (__byte_perm(a01, a23, 0x5410) + p.addc) ^ 0x80808080u;
+    w1 = (__byte_perm(a45, a67, 0x5410) + p.addc) ^ 0x80808080u;
+  } else {
+    w0 = pack4_offset(t, 0, p.addc);
+    w1 = pack4_offset(t, 4, p.addc);
+  }
   if (p.zero_all) { w0 = 0u; w1 = 0u; }
 }
 
 // Runs `body.template operator()<kMode, kHad32>()` for the operand's rounding mode and Hadamard block: the
 // per-chunk code is then free of mode and block-size tests (they cost more than a tenth of its instructions).
-template <bool kTrack, typename Body>
+// kClass: 0 = every rounding mode is compiled in, 1 = nearest only, 2 = the stochastic modes only (a kernel that
+// holds fewer bodies gets registers allotted for those alone)
+template <bool kTrack, int kClass, typename Body>
 __device__ __forceinline__ void dispatch_mode2(const QuantParams& p, int had_block, Body& body) {
   const int mode = (p.mode == HDQT_ROUND_NEAREST) ? 0 : (p.sr_magic ? 1 : 2);
   if (had_block == 32) {
-    if (mode == 0) body.template operator()<0, true, kTrack>();
-    else if (mode == 1) body.template operator()<1, true, kTrack>();
-    else body.template operator()<2, true, kTrack>();
+    if (kClass != 2 && mode == 0) body.template operator()<0, true, kTrack>();
+    else if (kClass != 1 && mode == 1) body.template operator()<1, true, kTrack>();
+    else if (kClass != 1 && mode == 2) body.template operator()<2, true, kTrack>();
   } else {
-    if (mode == 0) body.template operator()<0, false, kTrack>();
-    else if (mode == 1) body.template operator()<1, false, kTrack>();
-    else body.template operator()<2, false, kTrack>();
+    if (kClass != 2 && mode == 0) body.template operator()<0, false, kTrack>();
+    else if (kClass != 1 && mode == 1) body.template operator()<1, false, kTrack>();
+    else if (kClass != 1 && mode == 2) body.template operator()<2, false, kTrack>();
   }
 }
 // kTrack: the body also keeps the maximum magnitude of the transformed values it sees (delayed scaling)
-template <typename Body>
+template <int kClass = 0, typename Body>
 __device__ __forceinline__ void dispatch_mode(const QuantParams& p, int had_block, bool track, Body body) {
-  if (track) dispatch_mode2<true>(p, had_block, body);
-  else dispatch_mode2<false>(p, had_block, body);
+  if (track) dispatch_mode2<true, kClass>(p, had_block, body);
+  else dispatch_mode2<false, kClass>(p, had_block, body);
 }
 
 __device__ __forceinline__ QuantParams make_params(const QuantScale& qs, int bits, float clip, int mode,
@@ -520,7 +534,7 @@ quantize_kc_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
         for (int i = 0; i < 8; ++i) seen = max(seen, abs_bits(x[u][i]));
       }
       uint2 out;
-      quantize8<kMode>(x[u], p, (uint64_t)c, out.x, out.y);  // linear index of the chunk's first element is 8*c
+      quantize8<kMode, true>(x[u], p, (uint64_t)c, out.x, out.y);  // linear index of the chunk's first element is 8*c
       // codes are dense [rows, K_pad]: chunk c is bytes [8c, 8c+8)
       if (c < total) *reinterpret_cast<uint2*>(codes + (c << 3)) = out;
     }
@@ -591,7 +605,7 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
             for (int i = 0; i < 8; ++i) seen = max(seen, abs_bits(x[u][i]));
           }
           uint2 out;
-          quantize8<kMode>(x[u], p, g + u * g_step, out.x, out.y);
+          quantize8<kMode, true>(x[u], p, g + u * g_step, out.x, out.y);
           int ss = __dp4a((int)out.x, (int)out.x, 0);
           ss = __dp4a((int)out.y, (int)out.y, ss);
           ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
@@ -630,7 +644,7 @@ quantize_kc_norms_kernel(const __grid_constant__ QuantBatch b, const __grid_cons
           const bool valid = r[u] >= 0;
           const uint64_t g = valid ? (uint64_t)r[u] * (uint64_t)cpr + (uint64_t)(k0 >> 3) : 0u;
           uint2 out;
-          quantize8<kMode>(x[u], p, g, out.x, out.y);
+          quantize8<kMode, true>(x[u], p, g, out.x, out.y);
           int ss = __dp4a((int)out.x, (int)out.x, 0);
           ss = __dp4a((int)out.y, (int)out.y, ss);
           ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
@@ -708,6 +722,9 @@ absmax_ks_kernel(const __grid_constant__ QuantBatch b, int32_t* dev_status) {
   commit_partial_max(op, local_block, mx, dev_status);
 }
 
+// kClass: 1 = operands rounded to nearest, 2 = stochastically rounded operands (two kernels: this one runs at its
+// register limit, and the stochastic bodies would otherwise set the nearest body's register allotment)
+template <int kClass>
 __global__ void __launch_bounds__(kThreads, 3)
 quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__ PhiloxKeys keys,
                    int32_t* dev_status) {
@@ -754,7 +771,7 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
         float x8[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) x8[i] = x[8 * j + i];
-        quantize8<kMode>(x8, p, g0 + j, w[2 * j], w[2 * j + 1]);
+        quantize8<kMode, true>(x8, p, g0 + j, w[2 * j], w[2 * j + 1]);
         ss = __dp4a((int)w[2 * j], (int)w[2 * j], ss);
         ss = __dp4a((int)w[2 * j + 1], (int)w[2 * j + 1], ss);
       }
@@ -782,7 +799,7 @@ quantize_ks_kernel(const __grid_constant__ QuantBatch b, const __grid_constant__
     }
   }
   };
-  dispatch_mode(p, had_block, op.hist_out != nullptr, body);
+  dispatch_mode<kClass>(p, had_block, op.hist_out != nullptr, body);
   if (op.hist_out != nullptr) commit_history(op, local_block, seen, dev_status);
 }
 
@@ -920,14 +937,14 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
   }
   // ---- quantize pass: one launch per kernel variant
   const PhiloxKeys keys = make_philox_keys(seed);
-  for (int variant = 0; variant < 3; ++variant) {   // 0 = K contiguous, 1 = K contiguous + tile norms, 2 = K strided
+  for (int variant = 0; variant < 4; ++variant) {   // 0 = K contiguous, 1 = K contiguous + tile norms, 2 / 3 = K strided, nearest / stochastic
     QuantBatch b{};
     b.had_block = had_block;
     b.bits = bits;
     b.stream = philox_offset;
     int grid = 0;
     for (int i = 0; i < n_ops; ++i) {
-      const int v = (ops[i].ld_k != 1) ? 2 : (ops[i].tile_norms != nullptr ? 1 : 0);
+      const int v = (ops[i].ld_k != 1) ? (ops[i].mode == HDQT_ROUND_NEAREST ? 2 : 3) : (ops[i].tile_norms != nullptr ? 1 : 0);
       if (v != variant) continue;
       int g;
       if (variant == 0) {
@@ -947,7 +964,8 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
     if (b.n_ops == 0) continue;
     if (variant == 0) quantize_kc_kernel<<<grid, kThreads, 0, s>>>(b, keys, dev_status);
     else if (variant == 1) quantize_kc_norms_kernel<<<grid, kThreads, 0, s>>>(b, keys, dev_status);
-    else quantize_ks_kernel<<<grid, kThreads, 0, s>>>(b, keys, dev_status);
+    else if (variant == 2) quantize_ks_kernel<1><<<grid, kThreads, 0, s>>>(b, keys, dev_status);
+    else quantize_ks_kernel<2><<<grid, kThreads, 0, s>>>(b, keys, dev_status);
     if (cudaGetLastError() != cudaSuccess) return HDQT_ERR_CUDA;
   }
   return HDQT_OK;
