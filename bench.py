@@ -609,11 +609,14 @@ def run_training_report(args):
                           "config": {"workload": key}, "train_steps_per_s": rec}))
         return
     out = {}
-    for name, quantized in (("hdqt", True), ("fp32_torch", False)):
+    for name, quantized, extra in (("hdqt", True, {}),
+                                   ("hdqt_cuda_graph_delayed_scaling", True, {"graphed": True, "delayed": True}),
+                                   ("fp32_torch", False, {})):
+        hnn.reset_delayed_scaling()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         res = hnn.class_incremental_run(quantized, dev, steps_per_task=args.steps_per_task, seed=0,
-                                        log=lambda m, n=name: print(f"[{n}] {m}", file=sys.stderr))
+                                        log=lambda m, n=name: print(f"[{n}] {m}", file=sys.stderr), **extra)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
         res["steps_per_s_end_to_end"] = res["steps"] / dt
@@ -624,7 +627,8 @@ def run_training_report(args):
                       "config": {"workload": "class-incremental ResNet-18-width: 5 tasks x 20 synthetic classes, "
                                              f"{args.steps_per_task} steps per task, replay memory 2000, batch 64 new + 64 "
                                              "replayed, SGD lr 0.05 momentum 0.9 wd 2e-4, 4-bit inputs / 8-bit accumulators"},
-                      "hdqt": out["hdqt"], "fp32_torch": out["fp32_torch"]}))
+                      "hdqt": out["hdqt"], "hdqt_cuda_graph_delayed_scaling": out["hdqt_cuda_graph_delayed_scaling"],
+                      "fp32_torch": out["fp32_torch"]}))
 
 
 def free_port() -> int:

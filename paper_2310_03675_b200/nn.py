@@ -454,13 +454,15 @@ def cnn_train_step(model: ResNet18Width, opt, x, labels, step: int, n_seen: Opti
 
 def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_task: int = 20,
                           steps_per_task: int = 1000, batch: int = 128, memory: int = 2000, seed: int = 0,
-                          lr: float = 0.05, test_per_class: int = 20, blend: float = 0.2, log=None, **over):
+                          lr: float = 0.05, test_per_class: int = 20, blend: float = 0.2, log=None,
+                          graphed: bool = False, **over):
     """Plain-replay class-incremental training of the ResNet-18-width model on synthetic classes (paper
     Section 4: tasks arrive one after the other, a bounded memory of exemplars is replayed, the head grows with
     the classes seen; appendix: SGD lr 0.05, momentum 0.9, weight decay 2e-4, memory 2000).  Each batch mixes
     new-task samples and replayed exemplars 1:1.  `blend` is the weight of the class pattern in an image (the rest
     is uniform noise): small enough that the task is not solved trivially.  Returns a dict with the final accuracy over all classes seen,
-    the accuracy after each task and the number of steps taken."""
+    the accuracy after each task and the number of steps taken.  graphed=True replays each task's training step from
+    CUDA graphs (recorded anew per task, because the head grows)."""
     n_classes = tasks * classes_per_task
     patterns = class_patterns(n_classes, seed, device)
     torch.manual_seed(seed)
@@ -477,6 +479,7 @@ def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_t
         lo, hi = task * classes_per_task, (task + 1) * classes_per_task
         n_new = batch if mem_x is None else batch // 2
         model.train()
+        stepper = None
         for _ in range(steps_per_task):
             y = torch.randint(lo, hi, (n_new,), generator=g, device=device)
             x = synthetic_images(y, patterns, seed=seed + 1000 + step, blend=blend)
@@ -484,8 +487,19 @@ def class_incremental_run(quantized: bool, device, tasks: int = 5, classes_per_t
                 idx = torch.randint(0, mem_x.shape[0], (batch - n_new,), generator=g, device=device)
                 x = torch.cat([x, mem_x[idx]])
                 y = torch.cat([y, mem_y[idx]])
-            loss = cnn_train_step(model, opt, x, y, step, n_seen=hi)
-            step += 1
+            if not graphed:
+                loss = cnn_train_step(model, opt, x, y, step, n_seen=hi)
+                step += 1
+            elif stepper is None:
+                # (its three warm-up steps train on this first batch and count as steps of the task)
+                stepper = GraphedTrainStep(model, opt, x, y, forward=lambda inp, n=hi: model(inp, n),
+                                           base_step=(task + 1) * 1000003)
+                loss = stepper.losses[0]
+                step += 3
+            else:
+                loss = stepper(x, y)
+                step += 1
+        del stepper
         # exemplar memory: equal quota per class seen so far, random selection
         quota = memory // hi
         keep_x, keep_y = [], []

@@ -138,13 +138,17 @@ def test_resnet18_width_step_runs_and_learns():
     assert [p.shape for p in twin.parameters()] == [p.shape for p in model.parameters()]
 
 
-def test_class_incremental_loop_end_to_end_on_a_small_budget():
+@pytest.mark.parametrize("extra", [{}, {"graphed": True, "delayed": True}])
+def test_class_incremental_loop_end_to_end_on_a_small_budget(extra):
     """Two tasks of five classes, a few steps each: head growth, replay mixing, exemplar quota and evaluation run
-    through the quantized path; the accuracies are only required to be well-formed."""
+    through the quantized path (eager, and replayed from CUDA graphs recorded per task with delayed scaling); the
+    accuracies are only required to be well-formed."""
     from paper_2310_03675_b200 import nn as hnn
+    hnn.reset_delayed_scaling()
     res = hnn.class_incremental_run(True, torch.device("cuda"), tasks=2, classes_per_task=5, steps_per_task=6,
-                                    batch=32, memory=40, seed=0, test_per_class=4)
-    assert res["steps"] == 12 and len(res["accuracy_after_task"]) == 2
+                                    batch=32, memory=40, seed=0, test_per_class=4, **extra)
+    hnn.reset_delayed_scaling()
+    assert res["steps"] == (16 if extra else 12) and len(res["accuracy_after_task"]) == 2
     assert all(0.0 <= a <= 1.0 for a in res["accuracy_after_task"])
 
 
