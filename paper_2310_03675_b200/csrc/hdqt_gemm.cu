@@ -321,9 +321,12 @@ hdqt_status_t hdqt::gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const
     const int64_t unit = (tpa % 4 == 0) ? tpa : ((tpa % 2 == 0) ? 2 * tpa : 4 * tpa);   // lcm(4, tpa) tiles
     const int64_t units = tiles32 / unit;                                              // whole units in K
     int64_t want = sms / num_blocks;
-    // at least 8 stages per item (the fixed cost of an item is a few tiles' worth), at most `want` items
-    int64_t per_item = (units + want - 1) / want;
+    // at least 8 stages per item (the fixed cost of an item is a few tiles' worth, and its sums are added with one
+    // atomic per element), at most `want` items, and items of equal length (32 + 4 tiles is worse than 36 in one)
     const int64_t min_units = (32 + unit - 1) / unit;
+    if (want > units / min_units) want = units / min_units;
+    if (want < 1) want = 1;
+    int64_t per_item = (units + want - 1) / want;
     if (per_item < min_units) per_item = min_units;
     if (packed && per_item * unit > (int64_t)p.flush_every * tpa) per_item = (int64_t)p.flush_every * tpa / unit;
     const int64_t items = per_item > 0 ? (tiles32 + per_item * unit - 1) / (per_item * unit) : 1;

@@ -463,8 +463,31 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e
   const int64_t gn = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16;
   if (gn >= p.N) return;      // (warp-uniform) columns beyond the matrix: nothing to write
   if (job.atomic) {
-    // split-K: integer partial sums of this K range (the buffer was cleared before the launch)
-    if (gm < p.M) {
+    // split-K: integer partial sums of this K range (the buffer was cleared before the launch).  Through the box,
+    // like the stores: a warp-wide atomic then covers 8 rows x 16 consecutive words (8 memory transactions)
+    // instead of one word in each of 32 rows.
+    if (gn + 16 <= p.N) {
+      int4* dst = reinterpret_cast<int4*>(e.box + e.lane * 16);
+      const int rot = (e.lane >> 1) & 3;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) dst[(i + rot) & 3] = make_int4(val[4 * i], val[4 * i + 1], val[4 * i + 2], val[4 * i + 3]);
+      __syncwarp();
+      const int sub = e.lane >> 2, quad = e.lane & 3;
+#pragma unroll
+      for (int rr = 0; rr < 32; rr += 8) {
+        const int rloc = rr + sub;
+        const int4 v = *reinterpret_cast<const int4*>(e.box + rloc * 16 + ((quad + ((rloc >> 1) & 3)) & 3) * 4);
+        const int64_t grow = (int64_t)job.m0 + e.q * 32 + rloc;
+        if (grow < p.M) {
+          int* o = reinterpret_cast<int*>(p.out + grow * p.ld_out + gn + quad * 4);
+          if (v.x != 0) atomicAdd(o, v.x);
+          if (v.y != 0) atomicAdd(o + 1, v.y);
+          if (v.z != 0) atomicAdd(o + 2, v.z);
+          if (v.w != 0) atomicAdd(o + 3, v.w);
+        }
+      }
+      __syncwarp();
+    } else if (gm < p.M) {
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         if (gn + i < p.N && val[i] != 0) atomicAdd(reinterpret_cast<int*>(p.out + gm * p.ld_out + gn + i), val[i]);
