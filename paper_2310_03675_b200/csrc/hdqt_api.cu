@@ -23,6 +23,7 @@ hdqt_status_t check_quant_args(const float* src, int64_t rows, int64_t K, int64_
 }
 
 constexpr int64_t kMinBlocksForNorms = 32;
+constexpr int64_t kMinHarmonicForNorms = 512;   // M N / (M + N), see run_gemm
 
 struct OperandView {  // logical [rows, K] view of an operand with the contraction index as "K"
   const float* src;
@@ -186,7 +187,12 @@ hdqt_status_t run_gemm(const hdqt_gemm_desc_t* d, OperandView va, OperandView vb
     const int64_t p_max = tpa * 32 * code_max * code_max;
     const int64_t hi = (int64_t(1) << (d->acc_bits - 1)) - 1;
     const int64_t blocks = ((M + 127) / 128) * ((N + 255) / 256);
-    merge = (p_max > hi) && (blocks >= kMinBlocksForNorms);
+    // Tile norms (and with them the merging of clamp-free tiles) only where the GEMM outweighs the transform:
+    // its work grows with M N K, the quantize passes' with (M + N) K, so the ratio is M N / (M + N).  The norm
+    // output makes the quantize pass ~10 % slower and the GEMM carries the certificate bookkeeping; on the
+    // convolution layers of the CNN workload (N = 64 .. 512 output channels) that cost 8 % of a training step
+    // whatever the share of certified tiles, while the large square products gain up to 4x from merging.
+    merge = (p_max > hi) && (blocks >= kMinBlocksForNorms) && (M * N >= kMinHarmonicForNorms * (M + N));
   }
   int32_t* normsA = merge ? reinterpret_cast<int32_t*>(ws + L.norms_a) : nullptr;
   int32_t* normsB = merge ? reinterpret_cast<int32_t*>(ws + L.norms_b) : nullptr;
