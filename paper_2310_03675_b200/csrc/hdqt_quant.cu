@@ -918,14 +918,32 @@ hdqt_status_t launch_calibrate_quantize(const QuantOperand* ops, int n_ops, int3
     for (int i = 0; i < n_ops; ++i) {
       if ((ops[i].ld_k != 1) != (layout == 1) || ops[i].amax_in != nullptr || ops[i].hist_in != nullptr) continue;
       int g;
+      QuantOp cal = op[i];
       if (layout == 0) {
-        g = grid_for(op[i].rows * (op[i].K_pad >> 3), kThreads * kUnrollAbsmax, 4);
+        // Patch view of a convolution whose patches cover every input pixel: its 32-channel blocks are exactly the
+        // blocks of the activation tensor (each kh*kw times, plus all-zero padding blocks), so the maximum is taken
+        // over the tensor itself, [batch*H*W, C]: kh*kw times less to read, the same value bit for bit.
+        const ConvGeom& cg = ops[i].conv;
+        if (cg.enabled && cg.C % 32 == 0 && had_block == 32) {
+          const int64_t kh = ops[i].K / ((int64_t)cg.KW * cg.C);
+          const bool covered = cg.stride <= cg.KW && cg.stride <= kh &&
+                               (int64_t)(cg.Ho - 1) * cg.stride + kh - 1 - cg.pad >= cg.H - 1 &&
+                               (int64_t)(cg.Wo - 1) * cg.stride + cg.KW - 1 - cg.pad >= cg.W - 1;
+          if (covered) {
+            const int64_t batch = ops[i].rows / ((int64_t)cg.Ho * cg.Wo);
+            cal.conv.enabled = 0;
+            cal.rows = batch * cg.H * cg.W;
+            cal.K = cal.K_pad = cal.ld = cg.C;
+          }
+        }
+        g = grid_for(cal.rows * (cal.K_pad >> 3), kThreads * kUnrollAbsmax, 4);
       } else {
         g = grid_for(ks_items(op[i].rows, op[i].K_pad, op[i].rt_log2), 1, 3);
       }
       op[i].n_partials = g;
+      cal.n_partials = g;
       QuantOp& o = b.op[b.n_ops++];
-      o = op[i];
+      o = cal;
       o.first_block = grid;
       o.num_blocks = g;
       grid += g;
