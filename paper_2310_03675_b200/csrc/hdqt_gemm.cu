@@ -174,10 +174,10 @@ bool make_operand_map(CUtensorMap* map, const int8_t* base, int64_t rows, int64_
   return r == CUDA_SUCCESS;
 }
 
-template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false, bool kMerge = true>
+template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false, bool kMerge = true, bool kAtomic = true>
 hdqt_status_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, dim3 grid,
                              cudaStream_t s) {
-  auto kern = gemm_i8_tiled_kernel<kPacked, kShift, kTilesOut, kDeep, kMerge>;
+  auto kern = gemm_i8_tiled_kernel<kPacked, kShift, kTilesOut, kDeep, kMerge, kAtomic>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return cuda_failure(e, "cudaFuncSetAttribute(gemm)");
   kern<<<grid, GEMM_THREADS, SMEM_BYTES, s>>>(ma, mb, p);
@@ -395,11 +395,16 @@ hdqt_status_t hdqt::gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const
   const int64_t tiles_per_item = p.split_k > 1 ? (int64_t)p.split_kblocks * 4 / tpa : num_acc;
   const bool deep = packed && tiles_per_item >= 128 && tiles_per_item <= 256 * (int64_t)p.flush_every;
   if (packed && p.merge == 0) {      // no merged tiles in this launch: the kernel without the merged paths
-    st = deep ? launch_variant<true, false, false, true, false>(ma, mb, p, grid, s)
-              : launch_variant<true, false, false, false, false>(ma, mb, p, grid, s);
-  } else if (packed) {
-    st = deep ? launch_variant<true, false, false, true>(ma, mb, p, grid, s)
-              : launch_variant<true, false, false>(ma, mb, p, grid, s);
+    if (p.split_k > 1) {
+      st = deep ? launch_variant<true, false, false, true, false, true>(ma, mb, p, grid, s)
+                : launch_variant<true, false, false, false, false, true>(ma, mb, p, grid, s);
+    } else {
+      st = deep ? launch_variant<true, false, false, true, false, false>(ma, mb, p, grid, s)
+                : launch_variant<true, false, false, false, false, false>(ma, mb, p, grid, s);
+    }
+  } else if (packed) {       // (split-K work items only exist in launches that merge nothing)
+    st = deep ? launch_variant<true, false, false, true, true, false>(ma, mb, p, grid, s)
+              : launch_variant<true, false, false, false, true, false>(ma, mb, p, grid, s);
   }
   else st = acc_shift ? launch_variant<false, true, false>(ma, mb, p, grid, s)
                       : launch_variant<false, false, false>(ma, mb, p, grid, s);

@@ -456,13 +456,15 @@ __device__ __forceinline__ float dequant_scale(const GemmParams& p) {
 // kDirect: every thread stores its own row with 16-byte vector stores instead (no staging box, no warp syncs:
 // less code and fewer registers around a long main loop; less efficient stores, so only where the final pass is
 // rare: the long-contraction variant).
-template <bool kDirect = false>
+// kAtomic = false: the launch has no split-K work items; the atomic path is compiled out (the per-tile loops of the
+// clamp path lost 12 % to its mere presence in the kernel's code).
+template <bool kDirect = false, bool kAtomic = true>
 __device__ __forceinline__ void store_chunk(const GemmParams& p, const EpiCtx& e, const BlockJob& job, int c,
                                             int (&val)[16], bool parked, float scale, bool raw = false) {
   const int64_t gm = (int64_t)job.m0 + e.q * 32 + e.lane;
   const int64_t gn = (int64_t)job.n0 + e.grp * EPI_COLS + c * 16;
   if (gn >= p.N) return;      // (warp-uniform) columns beyond the matrix: nothing to write
-  if (job.atomic) {
+  if (kAtomic && job.atomic) {
     // split-K: integer partial sums of this K range (the buffer was cleared before the launch).  Through the box,
     // like the stores: a warp-wide atomic then covers 8 rows x 16 consecutive words (8 memory transactions)
     // instead of one word in each of 32 rows.
@@ -711,7 +713,7 @@ __device__ __forceinline__ void packed_accumulate(uint32_t (&S)[EPI_COLS / 2], u
 // kDeep (contractions of more than flush_every tiles, chosen by the host): a second set of 16-bit lanes takes the
 // high bytes of the lane sums every flush_every tiles (sum = low + 256 * high), so that nothing is parked in memory
 // for up to 256 * flush_every tiles; it costs 64 more registers, which is why it is a variant of its own.
-template <bool kDeep, bool kMerge = true>
+template <bool kDeep, bool kMerge = true, bool kAtomic = true>
 __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, BlockJob job, uint32_t& drain_par) {
   uint32_t S[EPI_COLS / 2];
   uint32_t Shi[kDeep ? EPI_COLS / 2 : 1];
@@ -836,7 +838,7 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
       if constexpr (kFast) {
         if (c < fast.chunks_inside) store_chunk_fast(fast, c, val, scale);   // (the rest lies beyond the matrix)
       } else {
-        store_chunk<kDeep>(p, e, job, c, val, parked, scale);
+        store_chunk<kDeep, kAtomic>(p, e, job, c, val, parked, scale);
       }
     }
   };

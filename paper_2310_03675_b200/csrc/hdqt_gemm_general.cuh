@@ -23,6 +23,7 @@ namespace {
 //          per register, clamp and add work on 16-bit lane pairs (half the ALU work per element).
 // kDeep:   with kPacked, for contractions longer than flush_every tiles: two-level lane sums (see epilogue_packed).
 // kMerge:  false = the launch merges no tiles; the merged paths are compiled out.
+// kAtomic: false = no split-K work items in the launch; the atomic store path is compiled out (packed variants).
 // otherwise: one 32-bit register per accumulator element, any b_a and r.
 
 struct TileInfo {                       // what the certificate warp publishes per output block
@@ -57,7 +58,7 @@ __device__ __forceinline__ void block_coords(const GemmParams& p, int i, int til
   }
 }
 
-template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false, bool kMerge = true>
+template <bool kPacked, bool kShift, bool kTilesOut, bool kDeep = false, bool kMerge = true, bool kAtomic = true>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
@@ -439,7 +440,7 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       job.n0 = tile_n * BN;
       bool ok;
       if (kMerge && job.n_clamp_tiles == 0 && job.n_merged > 0) ok = epilogue_merged_only<kDeep>(p, e, job, drain_par);
-      else if (kPacked) ok = epilogue_packed<kDeep, kMerge>(p, e, job, drain_par);
+      else if (kPacked) ok = epilogue_packed<kDeep, kMerge, kAtomic>(p, e, job, drain_par);
       else ok = epilogue_wide<kShift, kTilesOut>(p, e, job, drain_par);
       if (!ok) break;
       if (merge_mode == 1) {
