@@ -394,7 +394,8 @@ hdqt_status_t hdqt::gemm_i8_tiled_impl(const int8_t* Aq, const int8_t* Bq, const
   // run ~4 % faster for it (measured: 893 -> 931 TOPS at 8192^3, break-even near 128 tiles): used from 128 tiles.
   const int64_t tiles_per_item = p.split_k > 1 ? (int64_t)p.split_kblocks * 4 / tpa : num_acc;
   const bool deep = packed && tiles_per_item >= 128 && tiles_per_item <= 256 * (int64_t)p.flush_every;
-  if (packed && p.merge == 0) {      // no merged tiles in this launch: the kernel without the merged paths
+  if (packed && p.merge == 0 && (deep || tiles_per_item <= p.flush_every)) {
+    // no merged tiles in this launch, no work item that would have to park partial sums: the lean kernels
     if (p.split_k > 1) {
       st = deep ? launch_variant<true, false, false, true, false, true>(ma, mb, p, grid, s)
                 : launch_variant<true, false, false, false, false, true>(ma, mb, p, grid, s);

@@ -793,7 +793,7 @@ __device__ __forceinline__ bool epilogue_packed(const GemmParams& p, EpiCtx e, B
           S[i] &= 0x00FF00FFu;
         }
         n_deep += n_in_S;
-      } else {
+      } else if constexpr (kMerge) {     // (the merge-free instantiations never get work items that long)
         park_sums();
         n_in_S = 0;
         parked = true;
