@@ -111,6 +111,9 @@ gemm_i8_tiled_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   };
 
   if (threadIdx.x == 0) {
+    // the first TMA load would otherwise wait for its descriptor: fetch both while the CTA sets itself up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
