@@ -496,6 +496,34 @@ fixup_pair_blocks_kernel(const int8_t* __restrict__ Aq, const int8_t* __restrict
     __syncthreads();   // the corrections above and the conversion below use different thread-to-element maps
     // parked (now exact) integer sums -> fp32, lanes on consecutive columns; all loads first, so that
     // they are in flight together (each element is touched by this thread only)
+    const bool vec4 = ((p.ld_out & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) && (n0 + BN <= p.N) &&
+                      (m0 + FIX_ROWS <= p.M) && p.S_out == nullptr;      // block-uniform
+    if (vec4) {
+      // whole 64 x 256 item inside the matrix: 16-byte accesses, lane l on columns 4 l .. 4 l + 3 (+ 128)
+      int4 Sq[8][2];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        const float* row = p.out + (m0 + warp * 8 + r) * p.ld_out + n0 + 4 * lane;
+        Sq[r][0] = __ldcg(reinterpret_cast<const int4*>(row));
+        Sq[r][1] = __ldcg(reinterpret_cast<const int4*>(row + 128));
+      }
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        float* row = p.out + (m0 + warp * 8 + r) * p.ld_out + n0 + 4 * lane;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int64_t gn = n0 + 4 * lane + 128 * h;
+          float4 o;
+          o.x = finish1(p, __fmul_rn((float)Sq[r][h].x, scale), gn);
+          o.y = finish1(p, __fmul_rn((float)Sq[r][h].y, scale), gn + 1);
+          o.z = finish1(p, __fmul_rn((float)Sq[r][h].z, scale), gn + 2);
+          o.w = finish1(p, __fmul_rn((float)Sq[r][h].w, scale), gn + 3);
+          *reinterpret_cast<float4*>(row + 128 * h) = o;
+        }
+      }
+      __syncthreads();
+      continue;
+    }
     int Sv[8][8];
 #pragma unroll
     for (int r = 0; r < 8; ++r) {
